@@ -1,0 +1,129 @@
+/*
+ * hmar.h - C ABI of the B200 (sm_100a) library for HMAR's Markovian block-sparse attention.
+ *
+ * The operation (paper Sec. 4.1 "I/O-Aware Windowed Attention", Fig. attn-mask, App. B.3/B.4):
+ * exact softmax attention over the flattened multi-scale token sequence, where the K resolution
+ * scales of side_k x side_k tokens are laid out one after another (Sec. 3) and a token of scale k
+ * attends to every token of scales k-1 and k and to nothing else (Sec. 4.1, Markovian next-scale
+ * prediction); attention inside a scale is bidirectional (Sec. 3).  The first scale has no
+ * predecessor and attends to itself only.
+ *
+ * Conventions shared by every entry point
+ *   - n_k = side_lens[k]^2 tokens in scale k, L = sum n_k, tokens ordered scale after scale.
+ *   - Tensors are [B, H, rows, D] contiguous with D innermost, rows = L for the training calls.
+ *     D must be 64 (the paper's head dimension, App. B.4); anything else is HMAR_ERR_UNSUPPORTED.
+ *   - Entry points without suffix take bf16 tensors (raw 16-bit storage) and compute with bf16 tensor
+ *     core inputs, fp32 accumulation and fp32 softmax.  The `_f32` entry points are the debug build:
+ *     float tensors and plain fp32 FMA arithmetic everywhere.
+ *   - lse[b,h,i] = ln sum_j exp(softmax_scale * q_i . k_j) over the allowed j (natural log), fp32.
+ *   - Every tensor pointer is DEVICE memory owned by the caller, 16-byte aligned.  `side_lens` is a
+ *     HOST array read during the call.  The library allocates no per-call device memory; it owns a
+ *     small per-schedule plan cache (device work lists), created on the first call that uses a new
+ *     side_lens list and released by hmar_shutdown().  That first call synchronises an internal
+ *     stream and must therefore not be issued while `stream` is being captured.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *     They return HMAR_OK or a negative hmar_status.  Argument errors are found before any launch
+ *     and leave the outputs untouched.  No entry point throws, traps or synchronises the device.
+ *   - Every wait inside the kernels is bounded; a wait that runs out makes the kernel stop cleanly
+ *     and record a code that hmar_device_status() reports.
+ */
+#ifndef HMAR_H_
+#define HMAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HMAR_OK = 0,
+    HMAR_ERR_BAD_ARG = -1,        /* null pointer, non-positive size, misaligned pointer, too many scales */
+    HMAR_ERR_UNSUPPORTED = -2,    /* D != 64, or the device is not sm_100 */
+    HMAR_ERR_CUDA = -3,           /* a CUDA runtime / driver call failed */
+    HMAR_ERR_WORKSPACE = -4,      /* workspace missing or smaller than hmar_attn_bwd_workspace_bytes() */
+    HMAR_ERR_DEVICE_TIMEOUT = -5  /* a bounded wait inside a kernel ran out (see hmar_device_status) */
+} hmar_status;
+
+#define HMAR_MAX_SCALES 64
+
+/* Training forward (Sec. 4.1; App. B.4 benchmarks this pass).
+ *   q, k, v : [B,H,L,D] in;  out : [B,H,L,D] out;  lse : [B,H,L] fp32 out.
+ *   side_lens : host array of n_scales positive side lengths (any order of sizes is accepted). */
+int hmar_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse,
+                  int B, int H, int D, int n_scales, const int* side_lens,
+                  float softmax_scale, void* stream);
+int hmar_attn_fwd_f32(const float* q, const float* k, const float* v, float* out, float* lse,
+                      int B, int H, int D, int n_scales, const int* side_lens,
+                      float softmax_scale, void* stream);
+
+/* Bytes of caller-provided device scratch the backward needs for this problem (0 on bad arguments).
+ * The scratch holds delta = rowsum(dO o O) and the fp32 dQ accumulator; its contents on entry do not
+ * matter and are undefined on return. */
+size_t hmar_attn_bwd_workspace_bytes(int B, int H, int D, int n_scales, const int* side_lens);
+
+/* Training backward (App. B.4 benchmarks this pass; the gradient of the exact attention above).
+ *   in : q, k, v, out, dout [B,H,L,D]; lse [B,H,L] as written by the forward.
+ *   out: dq, dk, dv [B,H,L,D] (fully overwritten).
+ *   workspace : device scratch of at least hmar_attn_bwd_workspace_bytes() bytes, 256-byte aligned.
+ * dQ is accumulated with floating-point atomics, so its low-order bits may differ between runs. */
+int hmar_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                  const void* dout, void* dq, void* dk, void* dv,
+                  void* workspace, size_t workspace_bytes,
+                  int B, int H, int D, int n_scales, const int* side_lens,
+                  float softmax_scale, void* stream);
+int hmar_attn_bwd_f32(const float* q, const float* k, const float* v, const float* out, const float* lse,
+                      const float* dout, float* dq, float* dk, float* dv,
+                      void* workspace, size_t workspace_bytes,
+                      int B, int H, int D, int n_scales, const int* side_lens,
+                      float softmax_scale, void* stream);
+
+/* Inference step of one scale (Sec. 4.1: no prefix computation or KV cache beyond the previous
+ * scale; Sec. 4.2/4.4: every masked refinement sub-step of scale k sees scale k-1 and scale k).
+ *   q            : [B,H,n_cur,D]      queries of the current scale, n_cur = side_cur^2
+ *   k_prev,v_prev: [B,H,n_prev,D]     cached previous scale, n_prev = side_prev^2;
+ *                                     must be NULL iff side_prev == 0 (first scale)
+ *   k_cur, v_cur : [B,H,n_cur,D]      the current scale's own keys / values
+ *   out          : [B,H,n_cur,D];  lse : [B,H,n_cur] fp32 or NULL.
+ * Dense attention of q over (prev followed by cur); no mask inside the window. */
+int hmar_attn_scale_step(const void* q, const void* k_prev, const void* v_prev,
+                         const void* k_cur, const void* v_cur, void* out, float* lse,
+                         int B, int H, int D, int side_prev, int side_cur,
+                         float softmax_scale, void* stream);
+int hmar_attn_scale_step_f32(const float* q, const float* k_prev, const float* v_prev,
+                             const float* k_cur, const float* v_cur, float* out, float* lse,
+                             int B, int H, int D, int side_prev, int side_cur,
+                             float softmax_scale, void* stream);
+
+/* Host-side scale-block scheduler (Sec. 4.1: the kernel visits only the live blocks of the mask).
+ * Writes the work list of one head for `direction` 0 = forward (tiles of query rows, each with the
+ * contiguous key range it must visit) or 1 = backward (tiles of key rows with their query range).
+ * Each tile is 6 int32: {row_begin, row_count, partner_begin, partner_end, uniform, cost}; `uniform`
+ * is 1 when every row of the tile may see the whole partner range, 0 when rows carry their own
+ * bounds (several small scales packed into one tile).  Returns the number of tiles, or a negative
+ * hmar_status; writes at most max_tiles entries (pass NULL / 0 to query the count).  Host only. */
+int hmar_schedule_tiles(int n_scales, const int* side_lens, int direction,
+                        int32_t* tiles, int max_tiles);
+
+/* Blocks until the work queued on the current device has finished, then returns the code recorded
+ * by the kernels since the last call (HMAR_OK, or HMAR_ERR_DEVICE_TIMEOUT with *detail, if not NULL,
+ * telling which wait gave up) and clears it.  Diagnostics only; never needed for correct results. */
+int hmar_device_status(int* detail);
+
+/* Debug switch: nonzero routes the bf16 entry points through the plain SIMT kernels (the same ones
+ * the _f32 build uses) instead of the tensor-core kernels.  Returns the previous setting. */
+int hmar_debug_force_simt(int enable);
+
+/* Number of kernels the library has launched since it was loaded (all entry points, this process). */
+long long hmar_launch_count(void);
+
+/* Frees the plan cache on every device.  Safe to call more than once. */
+void hmar_shutdown(void);
+
+const char* hmar_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HMAR_H_ */

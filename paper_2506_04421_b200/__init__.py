@@ -1,0 +1,11 @@
+"""B200 (sm_100a) library for HMAR's Markovian block-sparse attention: Python binding.
+
+The product is the C-ABI shared library built from csrc/ (see include/hmar.h); this package
+only loads it and marshals torch device buffers into its calls.
+"""
+from .binding import (  # noqa: F401
+    HMAR_ERR_BAD_ARG, HMAR_ERR_CUDA, HMAR_ERR_DEVICE_TIMEOUT, HMAR_ERR_UNSUPPORTED,
+    HMAR_ERR_WORKSPACE, HMAR_OK, EXPORTED_SYMBOLS, HmarError, hmar_attn_bwd,
+    hmar_attn_bwd_workspace_bytes, hmar_attn_fwd, hmar_attn_scale_step, hmar_debug_force_simt,
+    hmar_device_status, hmar_launch_count, hmar_schedule_tiles, hmar_shutdown, lib, status_string,
+)

@@ -1,0 +1,193 @@
+"""ctypes binding of libhmar.so: argument marshalling only.
+
+Every function here has the name and argument order of the C entry point it wraps (see
+include/hmar.h). Tensors are torch CUDA tensors used purely as device buffers; all of the
+arithmetic runs inside the library's kernels. There is no CPU fallback: if the shared library
+is missing or fails to load, importing this module raises.
+"""
+import ctypes
+import os
+
+import torch
+
+from . import build as _build
+
+_LIB = None
+
+HMAR_OK = 0
+HMAR_ERR_BAD_ARG = -1
+HMAR_ERR_UNSUPPORTED = -2
+HMAR_ERR_CUDA = -3
+HMAR_ERR_WORKSPACE = -4
+HMAR_ERR_DEVICE_TIMEOUT = -5
+
+EXPORTED_SYMBOLS = (
+    "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd",
+    "hmar_attn_bwd_f32", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_schedule_tiles",
+    "hmar_device_status", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
+    "hmar_status_string",
+)
+
+
+class HmarError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+def lib():
+    """Load (building first if the sources are newer) the in-tree shared library."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = _build.LIB_PATH
+    if _build.needs_build():
+        path = _build.build()
+    L = ctypes.CDLL(path)
+    vp, ip, fp = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int), ctypes.c_float
+    i = ctypes.c_int
+    L.hmar_attn_fwd.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, ip, fp, vp]
+    L.hmar_attn_fwd_f32.argtypes = L.hmar_attn_fwd.argtypes
+    L.hmar_attn_bwd_workspace_bytes.argtypes = [i, i, i, i, ip]
+    L.hmar_attn_bwd_workspace_bytes.restype = ctypes.c_size_t
+    L.hmar_attn_bwd.argtypes = [vp] * 9 + [vp, ctypes.c_size_t, i, i, i, i, ip, fp, vp]
+    L.hmar_attn_bwd_f32.argtypes = L.hmar_attn_bwd.argtypes
+    L.hmar_attn_scale_step.argtypes = [vp] * 7 + [i, i, i, i, i, fp, vp]
+    L.hmar_attn_scale_step_f32.argtypes = L.hmar_attn_scale_step.argtypes
+    L.hmar_schedule_tiles.argtypes = [i, ip, i, ctypes.POINTER(ctypes.c_int32), i]
+    L.hmar_device_status.argtypes = [ip]
+    L.hmar_debug_force_simt.argtypes = [i]
+    L.hmar_launch_count.restype = ctypes.c_longlong
+    L.hmar_shutdown.restype = None
+    L.hmar_status_string.argtypes = [i]
+    L.hmar_status_string.restype = ctypes.c_char_p
+    for name in EXPORTED_SYMBOLS:
+        if getattr(L, name).restype is ctypes.c_int:
+            pass
+    _LIB = L
+    return L
+
+
+def status_string(status):
+    return lib().hmar_status_string(int(status)).decode()
+
+
+def _sides(side_lens):
+    arr = (ctypes.c_int * len(side_lens))(*[int(s) for s in side_lens])
+    return arr, len(side_lens)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _check(status, where):
+    if status != HMAR_OK:
+        raise HmarError(status, where)
+
+
+def _is_f32(t):
+    if t.dtype == torch.float32:
+        return True
+    if t.dtype == torch.bfloat16:
+        return False
+    raise TypeError("tensors must be bfloat16 or float32")
+
+
+def _need(*tensors):
+    for t in tensors:
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("tensors must be contiguous CUDA tensors")
+
+
+def hmar_attn_fwd(q, k, v, side_lens, softmax_scale, out=None, lse=None, stream=None):
+    """Training forward. q, k, v: [B,H,L,D]. Returns (out [B,H,L,D], lse [B,H,L] fp32)."""
+    _need(q, k, v, out, lse)
+    B, H, L, D = q.shape
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((B, H, L), dtype=torch.float32, device=q.device)
+    sides, n = _sides(side_lens)
+    fn = lib().hmar_attn_fwd_f32 if _is_f32(q) else lib().hmar_attn_fwd
+    _check(fn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, D, n, sides,
+              float(softmax_scale), _stream(stream)), "hmar_attn_fwd")
+    return out, lse
+
+
+def hmar_attn_bwd_workspace_bytes(B, H, D, side_lens):
+    sides, n = _sides(side_lens)
+    return int(lib().hmar_attn_bwd_workspace_bytes(B, H, D, n, sides))
+
+
+def hmar_attn_bwd(q, k, v, out, lse, dout, side_lens, softmax_scale, dq=None, dk=None, dv=None,
+                  workspace=None, stream=None):
+    """Training backward. Returns (dq, dk, dv), each [B,H,L,D]."""
+    _need(q, k, v, out, lse, dout, dq, dk, dv, workspace)
+    B, H, L, D = q.shape
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(q) if dk is None else dk
+    dv = torch.empty_like(q) if dv is None else dv
+    if workspace is None:
+        workspace = torch.empty(hmar_attn_bwd_workspace_bytes(B, H, D, side_lens), dtype=torch.uint8,
+                                device=q.device)
+    sides, n = _sides(side_lens)
+    fn = lib().hmar_attn_bwd_f32 if _is_f32(q) else lib().hmar_attn_bwd
+    _check(fn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv),
+              _ptr(workspace), workspace.numel() * workspace.element_size(), B, H, D, n, sides,
+              float(softmax_scale), _stream(stream)), "hmar_attn_bwd")
+    return dq, dk, dv
+
+
+def hmar_attn_scale_step(q, k_prev, v_prev, k_cur, v_cur, side_prev, side_cur, softmax_scale,
+                         out=None, lse=None, want_lse=True, stream=None):
+    """Inference step of one scale. q, k_cur, v_cur: [B,H,side_cur^2,D]; k_prev, v_prev:
+    [B,H,side_prev^2,D] or None when side_prev == 0. Returns (out, lse or None)."""
+    _need(q, k_prev, v_prev, k_cur, v_cur, out, lse)
+    B, H, n_cur, D = q.shape
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None and want_lse:
+        lse = torch.empty((B, H, n_cur), dtype=torch.float32, device=q.device)
+    fn = lib().hmar_attn_scale_step_f32 if _is_f32(q) else lib().hmar_attn_scale_step
+    _check(fn(_ptr(q), _ptr(k_prev), _ptr(v_prev), _ptr(k_cur), _ptr(v_cur), _ptr(out), _ptr(lse),
+              B, H, D, int(side_prev), int(side_cur), float(softmax_scale), _stream(stream)),
+           "hmar_attn_scale_step")
+    return out, lse
+
+
+def hmar_schedule_tiles(side_lens, direction):
+    """Work list of one head as a list of dicts (host only; needs no GPU)."""
+    sides, n = _sides(side_lens)
+    count = lib().hmar_schedule_tiles(n, sides, int(direction), None, 0)
+    if count < 0:
+        raise HmarError(count, "hmar_schedule_tiles")
+    buf = (ctypes.c_int32 * (6 * count))()
+    lib().hmar_schedule_tiles(n, sides, int(direction), buf, count)
+    keys = ("row_begin", "row_count", "partner_begin", "partner_end", "uniform", "cost")
+    return [dict(zip(keys, buf[6 * t:6 * t + 6])) for t in range(count)]
+
+
+def hmar_device_status():
+    """(status, detail) recorded by the kernels since the last call; synchronises the device."""
+    detail = ctypes.c_int(0)
+    status = lib().hmar_device_status(ctypes.byref(detail))
+    return status, detail.value
+
+
+def hmar_debug_force_simt(enable):
+    return lib().hmar_debug_force_simt(1 if enable else 0)
+
+
+def hmar_launch_count():
+    return int(lib().hmar_launch_count())
+
+
+def hmar_shutdown():
+    lib().hmar_shutdown()

@@ -1,0 +1,251 @@
+// C-ABI layer: argument validation, plan cache, dispatch to the kernel launchers.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <type_traits>
+#include <vector>
+
+#include "hmar_common.h"
+#include "launchers.h"
+#include "tc_launchers.h"
+
+namespace hmar {
+
+static std::atomic<long long> g_launches{0};
+static std::atomic<int> g_force_simt{0};
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// Device status word written by kernels whose bounded waits ran out: {code, detail}.
+__device__ int g_device_status[2];
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static int check_shape(int B, int H, int D) {
+    if (B <= 0 || H <= 0 || D <= 0) return HMAR_ERR_BAD_ARG;
+    if ((long long)B * H > 65535) return HMAR_ERR_BAD_ARG;   // heads map to gridDim.y
+    if (D != kHeadDim) return HMAR_ERR_UNSUPPORTED;
+    return HMAR_OK;
+}
+
+static int check_sides(int n_scales, const int* side_lens, ScaleTable* st) {
+    if (n_scales <= 0 || n_scales > HMAR_MAX_SCALES || side_lens == nullptr) return HMAR_ERR_BAD_ARG;
+    long long total = 0;
+    for (int s = 0; s < n_scales; ++s) {
+        if (side_lens[s] <= 0 || side_lens[s] > 4096) return HMAR_ERR_BAD_ARG;
+        total += (long long)side_lens[s] * side_lens[s];
+    }
+    if (total > (1 << 24)) return HMAR_ERR_BAD_ARG;
+    build_scale_table(n_scales, side_lens, st);
+    return HMAR_OK;
+}
+
+static int check_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return HMAR_ERR_CUDA; }
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+        cudaGetLastError();
+        return HMAR_ERR_CUDA;
+    }
+    return major == 10 ? HMAR_OK : HMAR_ERR_UNSUPPORTED;
+}
+
+static size_t round256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+static int* device_status_ptr() {
+    // One address per device; looked up on first use with that device current.
+    static std::mutex mu;
+    static std::map<int, int*> ptrs;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = ptrs.find(dev);
+    if (it != ptrs.end()) return it->second;
+    int* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_device_status) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    ptrs[dev] = p;
+    return p;
+}
+
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+static int fwd_impl(const T* q, const T* k, const T* v, T* out, float* lse, int B, int H, int D,
+                    int n_scales, const int* side_lens, float softmax_scale, void* stream, bool tensor_core) {
+    int rc = check_shape(B, H, D);
+    if (rc != HMAR_OK) return rc;
+    ScaleTable st;
+    rc = check_sides(n_scales, side_lens, &st);
+    if (rc != HMAR_OK) return rc;
+    if (!q || !k || !v || !out || !lse) return HMAR_ERR_BAD_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(lse))
+        return HMAR_ERR_BAD_ARG;
+    rc = check_device();
+    if (rc != HMAR_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        if (tensor_core && !g_force_simt.load())
+            return tc_fwd(q, k, v, out, lse, B * H, st, softmax_scale, device_status_ptr(), s);
+    }
+    return simt_fwd<T>(q, k, v, out, lse, B * H, st, softmax_scale, s) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
+}
+
+template <typename T>
+static int bwd_impl(const T* q, const T* k, const T* v, const T* out, const float* lse, const T* dout,
+                    T* dq, T* dk, T* dv, void* workspace, size_t workspace_bytes, int B, int H, int D,
+                    int n_scales, const int* side_lens, float softmax_scale, void* stream, bool tensor_core) {
+    int rc = check_shape(B, H, D);
+    if (rc != HMAR_OK) return rc;
+    ScaleTable st;
+    rc = check_sides(n_scales, side_lens, &st);
+    if (rc != HMAR_OK) return rc;
+    if (!q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return HMAR_ERR_BAD_ARG;
+    const void* ptrs[] = {q, k, v, out, lse, dout, dq, dk, dv};
+    for (const void* p : ptrs)
+        if (!aligned16(p)) return HMAR_ERR_BAD_ARG;
+    const size_t need = hmar_attn_bwd_workspace_bytes(B, H, D, n_scales, side_lens);
+    if (workspace == nullptr || workspace_bytes < need) return HMAR_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return HMAR_ERR_BAD_ARG;
+    rc = check_device();
+    if (rc != HMAR_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int L = st.start[st.n_scales];
+    float* delta = static_cast<float*>(workspace);
+    float* dq_acc = reinterpret_cast<float*>(static_cast<char*>(workspace) + round256((size_t)B * H * L * sizeof(float)));
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        if (tensor_core && !g_force_simt.load())
+            return tc_bwd(q, k, v, out, lse, dout, dq, dk, dv, delta, dq_acc, B * H, st, softmax_scale,
+                          device_status_ptr(), s);
+    }
+    (void)dq_acc;
+    return simt_bwd<T>(q, k, v, out, lse, dout, dq, dk, dv, delta, B * H, st, softmax_scale, s) == cudaSuccess
+               ? HMAR_OK : HMAR_ERR_CUDA;
+}
+
+template <typename T>
+static int step_impl(const T* q, const T* k_prev, const T* v_prev, const T* k_cur, const T* v_cur, T* out,
+                     float* lse, int B, int H, int D, int side_prev, int side_cur, float softmax_scale,
+                     void* stream, bool tensor_core) {
+    int rc = check_shape(B, H, D);
+    if (rc != HMAR_OK) return rc;
+    if (side_cur <= 0 || side_cur > 4096 || side_prev < 0 || side_prev > 4096) return HMAR_ERR_BAD_ARG;
+    if (!q || !k_cur || !v_cur || !out) return HMAR_ERR_BAD_ARG;
+    if ((side_prev == 0) != (k_prev == nullptr) || (k_prev == nullptr) != (v_prev == nullptr))
+        return HMAR_ERR_BAD_ARG;
+    const void* ptrs[] = {q, k_prev, v_prev, k_cur, v_cur, out, lse};
+    for (const void* p : ptrs)
+        if (!aligned16(p)) return HMAR_ERR_BAD_ARG;
+    rc = check_device();
+    if (rc != HMAR_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int n_prev = side_prev * side_prev, n_cur = side_cur * side_cur;
+    if constexpr (std::is_same<T, __nv_bfloat16>::value) {
+        if (tensor_core && !g_force_simt.load())
+            return tc_scale_step(q, k_prev, v_prev, k_cur, v_cur, out, lse, B * H, n_prev, n_cur, softmax_scale,
+                                 device_status_ptr(), s);
+    }
+    return simt_scale_step<T>(q, k_prev, v_prev, k_cur, v_cur, out, lse, B * H, n_prev, n_cur, softmax_scale, s)
+                   == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
+}
+
+}  // namespace hmar
+
+using namespace hmar;
+typedef __nv_bfloat16 bf16;
+
+extern "C" {
+
+int hmar_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse, int B, int H, int D,
+                  int n_scales, const int* side_lens, float softmax_scale, void* stream) {
+    return fwd_impl<bf16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, lse, B, H, D, n_scales,
+                          side_lens, softmax_scale, stream, true);
+}
+
+int hmar_attn_fwd_f32(const float* q, const float* k, const float* v, float* out, float* lse, int B, int H,
+                      int D, int n_scales, const int* side_lens, float softmax_scale, void* stream) {
+    return fwd_impl<float>(q, k, v, out, lse, B, H, D, n_scales, side_lens, softmax_scale, stream, false);
+}
+
+size_t hmar_attn_bwd_workspace_bytes(int B, int H, int D, int n_scales, const int* side_lens) {
+    ScaleTable st;
+    if (check_shape(B, H, D) != HMAR_OK || check_sides(n_scales, side_lens, &st) != HMAR_OK) return 0;
+    const size_t rows = (size_t)B * H * st.start[st.n_scales];
+    return round256(rows * sizeof(float)) + round256(rows * kHeadDim * sizeof(float));
+}
+
+int hmar_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                  const void* dout, void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
+                  int B, int H, int D, int n_scales, const int* side_lens, float softmax_scale, void* stream) {
+    return bwd_impl<bf16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (const bf16*)out, lse,
+                          (const bf16*)dout, (bf16*)dq, (bf16*)dk, (bf16*)dv, workspace, workspace_bytes, B, H,
+                          D, n_scales, side_lens, softmax_scale, stream, true);
+}
+
+int hmar_attn_bwd_f32(const float* q, const float* k, const float* v, const float* out, const float* lse,
+                      const float* dout, float* dq, float* dk, float* dv, void* workspace,
+                      size_t workspace_bytes, int B, int H, int D, int n_scales, const int* side_lens,
+                      float softmax_scale, void* stream) {
+    return bwd_impl<float>(q, k, v, out, lse, dout, dq, dk, dv, workspace, workspace_bytes, B, H, D, n_scales,
+                           side_lens, softmax_scale, stream, false);
+}
+
+int hmar_attn_scale_step(const void* q, const void* k_prev, const void* v_prev, const void* k_cur,
+                         const void* v_cur, void* out, float* lse, int B, int H, int D, int side_prev,
+                         int side_cur, float softmax_scale, void* stream) {
+    return step_impl<bf16>((const bf16*)q, (const bf16*)k_prev, (const bf16*)v_prev, (const bf16*)k_cur,
+                           (const bf16*)v_cur, (bf16*)out, lse, B, H, D, side_prev, side_cur, softmax_scale,
+                           stream, true);
+}
+
+int hmar_attn_scale_step_f32(const float* q, const float* k_prev, const float* v_prev, const float* k_cur,
+                             const float* v_cur, float* out, float* lse, int B, int H, int D, int side_prev,
+                             int side_cur, float softmax_scale, void* stream) {
+    return step_impl<float>(q, k_prev, v_prev, k_cur, v_cur, out, lse, B, H, D, side_prev, side_cur,
+                            softmax_scale, stream, false);
+}
+
+int hmar_schedule_tiles(int n_scales, const int* side_lens, int direction, int32_t* tiles, int max_tiles) {
+    ScaleTable st;
+    int rc = check_sides(n_scales, side_lens, &st);
+    if (rc != HMAR_OK) return rc;
+    if (direction != 0 && direction != 1) return HMAR_ERR_BAD_ARG;
+    std::vector<Tile> t = build_tiles(st, direction);
+    if (tiles != nullptr) {
+        const int n = (int)t.size() < max_tiles ? (int)t.size() : max_tiles;
+        for (int i = 0; i < n; ++i) std::memcpy(tiles + 6 * i, &t[i], sizeof(Tile));
+    }
+    return (int)t.size();
+}
+
+int hmar_device_status(int* detail) {
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return HMAR_ERR_CUDA; }
+    int host[2] = {0, 0};
+    if (cudaMemcpyFromSymbol(host, g_device_status, sizeof(host)) != cudaSuccess) { cudaGetLastError(); return HMAR_ERR_CUDA; }
+    const int zero[2] = {0, 0};
+    if (cudaMemcpyToSymbol(g_device_status, zero, sizeof(zero)) != cudaSuccess) { cudaGetLastError(); return HMAR_ERR_CUDA; }
+    if (detail) *detail = host[1];
+    return host[0] == 0 ? HMAR_OK : HMAR_ERR_DEVICE_TIMEOUT;
+}
+
+int hmar_debug_force_simt(int enable) { return g_force_simt.exchange(enable ? 1 : 0); }
+
+long long hmar_launch_count(void) { return g_launches.load(); }
+
+void hmar_shutdown(void) { tc_release_plans(); }
+
+const char* hmar_status_string(int status) {
+    switch (status) {
+        case HMAR_OK: return "ok";
+        case HMAR_ERR_BAD_ARG: return "bad argument";
+        case HMAR_ERR_UNSUPPORTED: return "unsupported head dimension or device";
+        case HMAR_ERR_CUDA: return "CUDA call failed";
+        case HMAR_ERR_WORKSPACE: return "workspace missing or too small";
+        case HMAR_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,43 @@
+// Shared host/device declarations of the HMAR attention library (internal).
+#pragma once
+#include <cstdint>
+#include <vector>
+#include "../../include/hmar.h"
+
+namespace hmar {
+
+constexpr int kHeadDim = 64;
+constexpr int kTileRows = 128;   // rows of one work tile (query rows forward, key rows backward)
+
+// Offsets of the scales in the flattened sequence; passed to kernels by value.
+struct ScaleTable {
+    int n_scales;
+    int start[HMAR_MAX_SCALES + 1];   // start[n_scales] == L
+};
+
+// One unit of work: `row_count` consecutive rows starting at `row_begin`, and the contiguous range
+// [partner_begin, partner_end) of the other operand those rows touch.
+// Forward: rows are queries, partners are keys.  Backward: rows are keys, partners are queries.
+struct Tile {
+    int32_t row_begin;
+    int32_t row_count;
+    int32_t partner_begin;
+    int32_t partner_end;
+    int32_t uniform;   // 1: every row sees the whole partner range; 0: rows have their own bounds
+    int32_t cost;      // number of kTileRows-wide partner tiles (for ordering)
+};
+
+// Forward bounds of query row `i` of scale s: keys [start[s-1], start[s+1]).
+// Backward bounds of key row `j` of scale s: queries [start[s], start[s+2]).
+void build_scale_table(int n_scales, const int* side_lens, ScaleTable* out);
+std::vector<Tile> build_tiles(const ScaleTable& st, int direction);
+
+#if defined(__CUDACC__)
+__device__ __forceinline__ int scale_of_row(const ScaleTable& st, int row) {
+    int s = 0;
+    while (s + 1 < st.n_scales && row >= st.start[s + 1]) ++s;
+    return s;
+}
+#endif
+
+}  // namespace hmar

@@ -1,0 +1,22 @@
+// Internal launcher prototypes shared between the C-ABI layer and the kernel files.
+#pragma once
+#include <cuda_runtime.h>
+#include "hmar_common.h"
+
+namespace hmar {
+
+void count_launch(int n);
+
+template <typename T>
+cudaError_t simt_fwd(const T* q, const T* k, const T* v, T* out, float* lse, int BH,
+                     const ScaleTable& st, float scale, cudaStream_t stream);
+template <typename T>
+cudaError_t simt_scale_step(const T* q, const T* k_prev, const T* v_prev, const T* k_cur, const T* v_cur,
+                            T* out, float* lse, int BH, int n_prev, int n_cur, float scale,
+                            cudaStream_t stream);
+template <typename T>
+cudaError_t simt_bwd(const T* q, const T* k, const T* v, const T* out, const float* lse, const T* dout,
+                     T* dq, T* dk, T* dv, float* delta, int BH, const ScaleTable& st, float scale,
+                     cudaStream_t stream);
+
+}  // namespace hmar

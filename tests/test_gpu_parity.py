@@ -1,0 +1,232 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 CPU oracle, element by element.
+
+Tolerances (written here, derived from the arithmetic):
+  * bf16 entry points: inputs are bf16 (shared with the oracle, so input rounding cancels), products
+    are exact in fp32, the softmax is fp32, P and dS are rounded to bf16 before the second matrix
+    product and the outputs are rounded to bf16 (relative 2^-9).  For N(0,1) inputs the outputs are
+    O(1), giving max |err| <= 2e-2 and mean |err| <= 2e-3 on out, dq, dk, dv; lse is fp32 and must
+    agree to 1e-3.
+  * fp32 debug entry points: <= 1e-5 on everything.
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2506_04421_b200 as hmar
+from oracle import hmar_oracle as orc
+from workloads import CONFIGS, scale_step_inputs, training_inputs
+from workloads.device import bulk_normal, to_device, training_tensors
+
+pytestmark = pytest.mark.gpu
+
+BF16_MAX, BF16_MEAN, LSE_TOL, F32_TOL = 2e-2, 2e-3, 1e-3, 1e-5
+
+
+def _err(gpu, ref):
+    d = np.abs(gpu.detach().double().cpu().numpy().reshape(ref.shape) - ref)
+    return float(d.max()), float(d.mean())
+
+
+def _assert_close(name, gpu, ref, is_f32):
+    mx, mean = _err(gpu, ref)
+    if is_f32:
+        assert mx <= F32_TOL, f"{name}: max abs err {mx:.3e} > {F32_TOL}"
+    else:
+        assert mx <= BF16_MAX, f"{name}: max abs err {mx:.3e} > {BF16_MAX}"
+        assert mean <= BF16_MEAN, f"{name}: mean abs err {mean:.3e} > {BF16_MEAN}"
+
+
+def _assert_lse(gpu, ref, is_f32):
+    mx, _ = _err(gpu, ref)
+    assert mx <= (F32_TOL if is_f32 else LSE_TOL), f"lse: max abs err {mx:.3e}"
+
+
+def _no_device_error():
+    status, detail = hmar.hmar_device_status()
+    assert status == hmar.HMAR_OK, f"device status {status} detail {detail:#x}"
+
+
+class _Wl:
+    """Ad-hoc workload for the edge-case side lists."""
+    def __init__(self, sides, B=1, H=2, seed=777):
+        self.B, self.H, self.D, self.side_lens, self.softmax_scale = B, H, 64, tuple(sides), 0.125
+        self.seed = seed + sum((i + 1) * s for i, s in enumerate(sides))
+        self.L = sum(s * s for s in sides)
+
+
+def _run_training(wl, dtype, gain=1.0, backward=True, simt=False):
+    is_f32 = dtype == torch.float32
+    q, k, v, do = training_inputs(wl, bf16=not is_f32, gain=gain)
+    prev = hmar.hmar_debug_force_simt(simt)
+    try:
+        tq, tk, tv, tdo = (to_device(x, wl.B, wl.H, dtype) for x in (q, k, v, do))
+        out, lse = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale)
+        ref_out, ref_lse = orc.attn_fwd(q, k, v, wl.side_lens, wl.softmax_scale)
+        _assert_close("out", out, ref_out, is_f32)
+        _assert_lse(lse, ref_lse, is_f32)
+        if backward:
+            dq, dk, dv = hmar.hmar_attn_bwd(tq, tk, tv, out, lse, tdo, wl.side_lens, wl.softmax_scale)
+            rq, rk, rv = orc.attn_bwd(q, k, v, do, wl.side_lens, wl.softmax_scale)
+            _assert_close("dq", dq, rq, is_f32)
+            _assert_close("dk", dk, rk, is_f32)
+            _assert_close("dv", dv, rv, is_f32)
+        _no_device_error()
+    finally:
+        hmar.hmar_debug_force_simt(prev)
+
+
+EDGE_SIDES = [(1,), (1, 1), (3, 11), (12, 12), (11, 12), (2, 1, 3, 1, 2), (12, 11, 1), (1, 2, 3, 4, 5, 6, 8, 10, 13, 16),
+              (16, 3, 17), (1, 23)]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_config1_tiny_fwd_bwd(dtype):
+    _run_training(CONFIGS["tiny"], dtype)
+
+
+@pytest.mark.parametrize("sides", EDGE_SIDES)
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_edge_side_lists_fwd_bwd(sides, dtype):
+    _run_training(_Wl(sides), dtype)
+
+
+@pytest.mark.parametrize("sides", [(1, 2, 3, 4), (3, 11), (1, 2, 3, 4, 5, 6, 8, 10, 13, 16)])
+def test_bf16_simt_fallback_kernels(sides):
+    _run_training(_Wl(sides), torch.bfloat16, simt=True)
+
+
+def test_large_logits_exercise_running_max():
+    # q scaled by 8: logits ~ N(0, 8^2), the running maximum moves often and P is peaked
+    _run_training(_Wl((1, 2, 3, 4, 6, 9, 13, 18)), torch.bfloat16, gain=8.0)
+    _run_training(_Wl((1, 2, 3, 4, 6, 9, 13, 18)), torch.float32, gain=8.0)
+
+
+def test_fp32_debug_build_512_shape_one_head():
+    _run_training(_Wl(CONFIGS["512_d24_train"].side_lens, B=1, H=1), torch.float32)
+
+
+def _sample_heads(BH, n=6):
+    rng = np.random.default_rng(BH)
+    picks = {0, BH - 1} | set(int(x) for x in rng.integers(0, BH, size=n))
+    return sorted(picks)
+
+
+@pytest.mark.parametrize("name", ["256_d16_fwd", "256_d30_train", "512_d24_train"])
+def test_full_size_configs_sampled_heads(name):
+    """Configs 2-4 at their full sizes, in the launch shape the benchmark times; the oracle checks
+    a sample of heads (always the first and the last) element by element."""
+    wl = CONFIGS[name]
+    heads = _sample_heads(wl.B * wl.H, 6 if wl.L < 1000 else 3)
+    backward = "bwd" in wl.passes
+    dev, host = training_tensors(wl, heads, with_dout=backward)
+    out, lse = hmar.hmar_attn_fwd(dev["q"], dev["k"], dev["v"], wl.side_lens, wl.softmax_scale)
+    idx = torch.as_tensor(heads, device="cuda")
+    ref_out, ref_lse = orc.attn_fwd(host["q"], host["k"], host["v"], wl.side_lens, wl.softmax_scale)
+    _assert_close("out", out.view(-1, wl.L, wl.D)[idx], ref_out, False)
+    _assert_lse(lse.view(-1, wl.L)[idx], ref_lse, False)
+    # properties that hold for every head: finite outputs, |out| bounded by max |v| of the head
+    assert torch.isfinite(out).all() and torch.isfinite(lse).all()
+    assert (out.float().abs().amax(dim=(2, 3)) <= dev["v"].float().abs().amax(dim=(2, 3)) * 1.01).all()
+    if backward:
+        dq, dk, dv = hmar.hmar_attn_bwd(dev["q"], dev["k"], dev["v"], out, lse, dev["dout"], wl.side_lens,
+                                        wl.softmax_scale)
+        rq, rk, rv = orc.attn_bwd(host["q"], host["k"], host["v"], host["dout"], wl.side_lens, wl.softmax_scale)
+        for nm, g, r in (("dq", dq, rq), ("dk", dk, rk), ("dv", dv, rv)):
+            assert torch.isfinite(g).all()
+            _assert_close(nm, g.view(-1, wl.L, wl.D)[idx], r, False)
+        # column sums of dV equal column sums of dO for every head (rows of P sum to one)
+        s_dv = dv.float().sum(dim=2)
+        s_do = dev["dout"].float().sum(dim=2)
+        assert (s_dv - s_do).abs().max().item() < 0.5     # sums of L bf16-rounded terms
+    _no_device_error()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_scale_step_small_batch_all_scales(dtype):
+    wl = CONFIGS["512_d24_infer"]
+    is_f32 = dtype == torch.float32
+    heads = [0, 1, 700, wl.B * wl.H - 1]
+    B, H = 2, 2
+    for s, side in enumerate(wl.side_lens):
+        for sub in (0, 3):
+            q, kp, vp, kc, vc = scale_step_inputs(wl, s, sub, bf16=not is_f32, heads=heads)
+            dev = [None if x is None else to_device(x, B, H, dtype) for x in (q, kp, vp, kc, vc)]
+            side_prev = wl.side_lens[s - 1] if s else 0
+            out, lse = hmar.hmar_attn_scale_step(*dev, side_prev, side, wl.softmax_scale)
+            ref_out, ref_lse = orc.scale_step(q, kp, vp, kc, vc, wl.softmax_scale)
+            _assert_close(f"out[scale {s}]", out, ref_out, is_f32)
+            _assert_lse(lse, ref_lse, is_f32)
+            out2, none = hmar.hmar_attn_scale_step(*dev, side_prev, side, wl.softmax_scale, want_lse=False)
+            assert none is None and torch.equal(out2, out)
+    _no_device_error()
+
+
+def test_scale_step_full_batch_last_scales_sampled_heads():
+    """Config 5 at B=64, H=24 for the three largest scales; sampled heads against the oracle."""
+    wl = CONFIGS["512_d24_infer"]
+    BH = wl.B * wl.H
+    heads = _sample_heads(BH, 2)
+    idx = torch.as_tensor(heads, device="cuda")
+    for s in (0, 7, 8, 9):
+        side, side_prev = wl.side_lens[s], (wl.side_lens[s - 1] if s else 0)
+        host = scale_step_inputs(wl, s, 1, bf16=True, heads=heads)
+        dev = []
+        for sid, h in enumerate(host):
+            if h is None:
+                dev.append(None)
+                continue
+            t = bulk_normal(wl.seed + s, sid, wl.B, wl.H, h.shape[1], wl.D)
+            t.view(BH, h.shape[1], wl.D)[idx] = torch.from_numpy(h).to(device="cuda", dtype=torch.bfloat16)
+            dev.append(t)
+        out, lse = hmar.hmar_attn_scale_step(*dev, side_prev, side, wl.softmax_scale)
+        ref_out, ref_lse = orc.scale_step(*host, wl.softmax_scale)
+        _assert_close(f"out[scale {s}]", out.view(BH, -1, wl.D)[idx], ref_out, False)
+        _assert_lse(lse.view(BH, -1)[idx], ref_lse, False)
+        assert torch.isfinite(out).all()
+    _no_device_error()
+
+
+def test_scale_step_matches_training_forward_rows():
+    """The inference step of scale k equals the scale-k rows of the training forward (same kernels'
+    arithmetic, different entry point)."""
+    wl = _Wl((2, 5, 12, 3))
+    q, k, v, _ = training_inputs(wl, bf16=True)
+    tq, tk, tv = (to_device(x, wl.B, wl.H, torch.bfloat16) for x in (q, k, v))
+    out, lse = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale)
+    starts = np.concatenate([[0], np.cumsum([s * s for s in wl.side_lens])])
+    for s, side in enumerate(wl.side_lens):
+        cur = slice(starts[s], starts[s + 1])
+        prev = slice(starts[s - 1], starts[s]) if s else None
+        o, l = hmar.hmar_attn_scale_step(
+            tq[:, :, cur].contiguous(),
+            None if prev is None else tk[:, :, prev].contiguous(),
+            None if prev is None else tv[:, :, prev].contiguous(),
+            tk[:, :, cur].contiguous(), tv[:, :, cur].contiguous(),
+            wl.side_lens[s - 1] if s else 0, side, wl.softmax_scale)
+        assert (o.float() - out[:, :, cur].float()).abs().max().item() <= 1e-2
+        assert (l - lse[:, :, cur]).abs().max().item() <= 1e-4
+
+
+def test_bad_workspace_is_rejected():
+    wl = CONFIGS["tiny"]
+    q, k, v, do = training_inputs(wl)
+    tq, tk, tv, tdo = (to_device(x, wl.B, wl.H, torch.bfloat16) for x in (q, k, v, do))
+    out, lse = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale)
+    small = torch.empty(64, dtype=torch.uint8, device="cuda")
+    with pytest.raises(hmar.HmarError) as e:
+        hmar.hmar_attn_bwd(tq, tk, tv, out, lse, tdo, wl.side_lens, wl.softmax_scale, workspace=small)
+    assert e.value.status == hmar.HMAR_ERR_WORKSPACE
+
+
+def test_repeat_calls_are_stable():
+    wl = _Wl((1, 2, 3, 4, 6, 9, 13))
+    q, k, v, do = training_inputs(wl)
+    tq, tk, tv, tdo = (to_device(x, wl.B, wl.H, torch.bfloat16) for x in (q, k, v, do))
+    o1, l1 = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale)
+    o2, l2 = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale)
+    assert torch.equal(o1, o2) and torch.equal(l1, l2)     # the forward is deterministic
+    g1 = hmar.hmar_attn_bwd(tq, tk, tv, o1, l1, tdo, wl.side_lens, wl.softmax_scale)
+    g2 = hmar.hmar_attn_bwd(tq, tk, tv, o1, l1, tdo, wl.side_lens, wl.softmax_scale)
+    assert torch.equal(g1[1], g2[1]) and torch.equal(g1[2], g2[2])        # dk, dv deterministic
+    assert (g1[0].float() - g2[0].float()).abs().max().item() <= 2e-2     # dq: atomics, order may differ
+    assert hmar.hmar_launch_count() > 0

@@ -1,0 +1,105 @@
+"""Host logic: the scale-block scheduler against the oracle's explicit mask, the C ABI's symbol
+table against include/hmar.h, and argument validation (which runs before any device is touched)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2506_04421_b200 as hmar
+from oracle import hmar_oracle as orc
+from workloads import CONFIGS
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+SIDE_LISTS = [
+    (1,), (1, 1), (3, 11), (12, 12), (1, 2, 3, 4), (2, 1, 3, 1, 2), (11, 12), (12, 11, 1),
+    CONFIGS["256_d16_fwd"].side_lens, CONFIGS["512_d24_train"].side_lens, (1, 2, 4, 8, 16, 32, 64),
+]
+
+
+@pytest.mark.parametrize("sides", SIDE_LISTS)
+@pytest.mark.parametrize("direction", [0, 1])
+def test_tiles_cover_exactly_the_live_blocks(sides, direction):
+    M = orc.hmar_mask(sides)
+    if direction == 1:
+        M = M.T            # rows = keys, columns = the queries that see them
+    L = M.shape[0]
+    tiles = hmar.hmar_schedule_tiles(sides, direction)
+    seen = np.zeros(L, dtype=int)
+    for t in tiles:
+        r0, rc = t["row_begin"], t["row_count"]
+        assert 0 < rc <= 128 and 0 <= r0 and r0 + rc <= L
+        seen[r0:r0 + rc] += 1
+        sub = M[r0:r0 + rc]
+        cols = np.nonzero(sub.any(axis=0))[0]
+        # the partner range is the tight hull of what the tile's rows may touch
+        assert cols.min() == t["partner_begin"] and cols.max() + 1 == t["partner_end"]
+        # every row's support is one contiguous run inside that range
+        for row in sub:
+            idx = np.nonzero(row)[0]
+            assert idx[-1] - idx[0] + 1 == len(idx)
+        full = bool(sub[:, t["partner_begin"]:t["partner_end"]].all())
+        assert full == bool(t["uniform"])
+        assert t["cost"] == -(-(t["partner_end"] - t["partner_begin"]) // 128)
+    assert (seen == 1).all()              # every row in exactly one tile
+    costs = [t["cost"] for t in tiles]
+    assert costs == sorted(costs, reverse=True)
+
+
+def test_tile_counts_for_paper_shapes():
+    # 512x512 schedule: scales 1-5 packed (66 rows), scale 6 alone, then 2+3+5+8 full-scale tiles
+    t = hmar.hmar_schedule_tiles(CONFIGS["512_d24_train"].side_lens, 0)
+    assert len(t) == 20 and sum(x["uniform"] == 0 for x in t) == 1
+    t = hmar.hmar_schedule_tiles(CONFIGS["256_d16_fwd"].side_lens, 0)
+    assert len(t) == 7
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "hmar.h")).read()
+    declared = set(re.findall(r"\b(hmar_[a-z0-9_]+)\s*\(", header))
+    declared -= {"hmar_status"}
+    assert declared == set(hmar.EXPORTED_SYMBOLS)
+    L = hmar.lib()
+    for name in declared:
+        assert getattr(L, name) is not None
+
+
+def _call_fwd(q=1 << 12, k=1 << 12, v=1 << 12, out=1 << 12, lse=1 << 12, B=1, H=1, D=64, sides=(1, 2)):
+    arr = (ctypes.c_int * max(len(sides), 1))(*sides)
+    vp = ctypes.c_void_p
+    return hmar.lib().hmar_attn_fwd(vp(q), vp(k), vp(v), vp(out), vp(lse), B, H, D, len(sides), arr,
+                                    0.125, None)
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    # pointers are fake but never dereferenced: validation fails first
+    assert _call_fwd(q=0) == hmar.HMAR_ERR_BAD_ARG
+    assert _call_fwd(q=(1 << 12) + 4) == hmar.HMAR_ERR_BAD_ARG          # misaligned
+    assert _call_fwd(B=0) == hmar.HMAR_ERR_BAD_ARG
+    assert _call_fwd(D=128) == hmar.HMAR_ERR_UNSUPPORTED
+    assert _call_fwd(sides=()) == hmar.HMAR_ERR_BAD_ARG
+    assert _call_fwd(sides=(1, 0, 2)) == hmar.HMAR_ERR_BAD_ARG
+    assert _call_fwd(sides=(1, -3)) == hmar.HMAR_ERR_BAD_ARG
+    assert _call_fwd(sides=tuple([1] * 65)) == hmar.HMAR_ERR_BAD_ARG
+    assert _call_fwd(B=70000) == hmar.HMAR_ERR_BAD_ARG
+    assert hmar.hmar_attn_bwd_workspace_bytes(1, 1, 32, (1, 2)) == 0
+    assert hmar.hmar_attn_bwd_workspace_bytes(2, 3, 64, (1, 2)) >= 2 * 3 * 5 * (64 + 1) * 4
+    with pytest.raises(hmar.HmarError):
+        hmar.hmar_schedule_tiles((1, 0), 0)
+    assert hmar.status_string(hmar.HMAR_ERR_WORKSPACE) == "workspace missing or too small"
+    vp = ctypes.c_void_p
+    # scale step: k_prev must be NULL exactly when side_prev == 0
+    f = hmar.lib().hmar_attn_scale_step
+    p = vp(1 << 12)
+    assert f(p, None, None, p, p, p, None, 1, 1, 64, 2, 3, 0.125, None) == hmar.HMAR_ERR_BAD_ARG
+    assert f(p, p, p, p, p, p, None, 1, 1, 64, 0, 3, 0.125, None) == hmar.HMAR_ERR_BAD_ARG
+    assert f(p, p, p, p, p, p, None, 1, 1, 64, 2, 0, 0.125, None) == hmar.HMAR_ERR_BAD_ARG
+
+
+def test_valid_call_without_a_device_fails_loudly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    assert _call_fwd() in (hmar.HMAR_ERR_CUDA, hmar.HMAR_ERR_UNSUPPORTED)
