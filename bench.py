@@ -1,0 +1,300 @@
+#!/usr/bin/env python
+"""Benchmark of the HMAR Markovian block-sparse attention path on B200.
+
+A step is one pass of the whole hot path on the 512x512 HMAR-d24 training shape (B=16, H=24,
+L=2240, D=64): forward, then backward, through the C ABI on bf16 device tensors.  The metric is
+useful TFLOP/s: only the unmasked (query, key) pairs count, 4*pairs*D for the forward and
+10*pairs*D for the backward, per head.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same shape on its own tensors
+(the path has no exchange step: independent replicas, weak scaling); the time is the maximum over
+ranks.  `--impl reference` times the CPU oracle, as it stands, on a bounded sample of heads.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+WORKLOAD = "512_d24_train"
+METRIC = "useful_tflops_fwd_bwd_512x512_d24"
+UNIT = "TFLOP/s"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (None until a capture exists for the current kernel).
+NCU_TRAFFIC_BYTES = {"hmar_bwd": None, "hmar_fwd": None}
+
+
+def pairs_per_head(side_lens):
+    n = [s * s for s in side_lens]
+    return sum(n[i] * (n[i] + (n[i - 1] if i else 0)) for i in range(len(n)))
+
+
+def useful_flops(wl):
+    p = pairs_per_head(wl.side_lens) * wl.B * wl.H * wl.D
+    return 4 * p, 10 * p
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_tflops": d["bf16_tflops"], "bf16_tflops_sustained": d.get("bf16_tflops_sustained"),
+                "hbm_gbs": d["hbm_gbs"], "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, sm_max, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                sm_max.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower() == "active":
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(sm_max)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def time_oracle(wl, n_heads, steps, warmup):
+    """Times the CPU oracle (forward + backward) on `n_heads` heads of the workload per step."""
+    from threadpoolctl import threadpool_info
+
+    from oracle import hmar_oracle as orc
+    from workloads import training_inputs
+    heads = sorted({0, wl.B * wl.H - 1} | set(range(1, n_heads - 1)))[:n_heads]
+    q, k, v, do = training_inputs(wl, bf16=True, heads=heads)
+    times = []
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        orc.attn_fwd(q, k, v, wl.side_lens, wl.softmax_scale)
+        orc.attn_bwd(q, k, v, do, wl.side_lens, wl.softmax_scale)
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+    flops = 14 * pairs_per_head(wl.side_lens) * wl.D * len(heads)
+    cores = max([p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"] or [1])
+    sec = float(np.mean(times))
+    return {"value": flops / sec / 1e12, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": f"{len(heads)} of {wl.B * wl.H} heads (first, last and the heads between), fwd+bwd, "
+                      f"{sec * 1e3:.0f} ms per sample; numpy fp64 with an explicit {wl.L}x{wl.L} mask"}, sec
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_heads = 4
+    base, sec = time_oracle(wl, n_heads, args.steps, min(args.warmup, 1))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": base["value"], "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": min(args.warmup, 1), "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "B": wl.B, "H": wl.H, "L": wl.L, "D": wl.D,
+                   "side_lens": list(wl.side_lens), "note": "CPU oracle; each step is the bounded sample below"},
+        "cpu_baseline": base,
+        "e2e": {"value": base["value"], "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2506_04421_b200 as hmar
+    from workloads.device import bulk_normal
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the HMAR library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    B, H, L, D = wl.B, wl.H, wl.L, wl.D
+    sides, scale = wl.side_lens, wl.softmax_scale
+    seed = wl.seed + 1000 * rank
+    q, k, v, do = (bulk_normal(seed, i, B, H, L, D, torch.bfloat16, dev) for i in range(4))
+    out = torch.empty_like(q)
+    lse = torch.empty((B, H, L), dtype=torch.float32, device=dev)
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    ws = torch.empty(hmar.hmar_attn_bwd_workspace_bytes(B, H, D, sides), dtype=torch.uint8, device=dev)
+
+    def step():
+        hmar.hmar_attn_fwd(q, k, v, sides, scale, out=out, lse=lse)
+        hmar.hmar_attn_bwd(q, k, v, out, lse, do, sides, scale, dq=dq, dk=dk, dv=dv, workspace=ws)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+
+    # ---- device-resident timing: K steps between two events, plus per-call events for the roofline
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    launches0 = hmar.hmar_launch_count()
+    barrier()
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_begin.record()
+    for i in range(args.steps):
+        ev[i][0].record()
+        hmar.hmar_attn_fwd(q, k, v, sides, scale, out=out, lse=lse)
+        ev[i][1].record()
+        hmar.hmar_attn_bwd(q, k, v, out, lse, do, sides, scale, dq=dq, dk=dk, dv=dv, workspace=ws)
+        ev[i][2].record()
+    t_end.record()
+    barrier()
+    launches = hmar.hmar_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    total_ms = t_begin.elapsed_time(t_end)
+    fwd_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    bwd_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    status, detail = hmar.hmar_device_status()
+    if status != 0:
+        raise RuntimeError(f"device status {status} detail {detail:#x}")
+
+    # ---- end to end: pinned host tensors in, results back to the host, inside the timed region
+    hq, hk, hv, hdo = (t.cpu().pin_memory() for t in (q, k, v, do))
+    h_out, h_dq, h_dk, h_dv = (torch.empty_like(hq).pin_memory() for _ in range(4))
+    h_lse = torch.empty((B, H, L), dtype=torch.float32).pin_memory()
+
+    def e2e_step():
+        q.copy_(hq, non_blocking=True)
+        k.copy_(hk, non_blocking=True)
+        v.copy_(hv, non_blocking=True)
+        do.copy_(hdo, non_blocking=True)
+        step()
+        h_out.copy_(out, non_blocking=True)
+        h_lse.copy_(lse, non_blocking=True)
+        h_dq.copy_(dq, non_blocking=True)
+        h_dk.copy_(dk, non_blocking=True)
+        h_dv.copy_(dv, non_blocking=True)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    times = torch.tensor([total_ms, e2e_ms, fwd_ms, bwd_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms, fwd_ms, bwd_ms = times.tolist()
+    ms_per_step = total_ms / args.steps
+    f_fwd, f_bwd = useful_flops(wl)
+    value = world * (f_fwd + f_bwd) / (ms_per_step * 1e-3) / 1e12
+    e2e_value = world * (f_fwd + f_bwd) / (e2e_ms * 1e-3) / 1e12
+
+    if rank == 0:
+        peaks = measured_peaks()
+        bwd_tf = f_bwd / (bwd_ms * 1e-3) / 1e12
+        fwd_tf = f_fwd / (fwd_ms * 1e-3) / 1e12
+        cpu_base, _ = time_oracle(wl, 24, 2, 0)
+        elem = 2 * B * H * L * D
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "B": B, "H": H, "L": L, "D": D, "side_lens": list(sides),
+                       "softmax_scale": scale, "passes": "fwd+bwd", "parallelism": f"replicas x{world}",
+                       "l2": "tensors larger than L2 (8 x 110 MB + 446 MB scratch per step), no flush"},
+            "fraction_of_peak": {"burst": value / world / peaks["bf16_tflops"],
+                                 "sustained": value / world / (peaks["bf16_tflops_sustained"] or float("nan")),
+                                 "nominal_2250": value / world / 2250.0, "peaks": peaks["source"]},
+            "phases": {"fwd_ms": fwd_ms, "bwd_ms": bwd_ms, "fwd_tflops": fwd_tf, "bwd_tflops": bwd_tf},
+            "roofline": {"bound": "tensor", "kernel": "backward call (delta + main + dq convert)",
+                         "achieved": bwd_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": bwd_tf / peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst",
+                         "traffic": NCU_TRAFFIC_BYTES["hmar_bwd"]},
+            "cpu_baseline": cpu_base,
+            "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": 4 * elem, "d2h_bytes_per_step": 4 * elem + 4 * B * H * L},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    from workloads import CONFIGS
+    wl = CONFIGS[WORKLOAD]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()
