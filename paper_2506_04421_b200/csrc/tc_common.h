@@ -1,0 +1,36 @@
+// Argument structures shared by the tensor-core kernels and their host-side dispatch (internal).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include "hmar_common.h"
+
+namespace hmar {
+
+// Device form of a forward work tile: query rows [row_begin, row_begin + row_count) and up to two key
+// segments (second one used by the inference step only: previous scale, then current scale).
+struct FwdWork {
+    int32_t row_begin, row_count;
+    int32_t s0_begin, s0_end;
+    int32_t s1_begin, s1_end;
+    int32_t uniform;
+    int32_t pad;
+};
+
+struct FwdArgs {
+    const FwdWork* work;     // n_work tiles per head; nullptr = inference step (tiles derived in-kernel)
+    int n_work;
+    int n_q_rows;            // rows per head of q / out / lse
+    int n0, n1;              // inference step: rows of the previous / current scale's keys
+    float scale_log2;        // softmax_scale * log2(e)
+    __nv_bfloat16* out;
+    float* lse;              // may be nullptr
+    int* status;             // device status word {code, detail}, may be nullptr
+    ScaleTable st;
+};
+
+size_t fwd_tc_smem_bytes();
+cudaError_t launch_fwd_tc(const CUtensorMap& q, const CUtensorMap& k0, const CUtensorMap& v0, const CUtensorMap& k1,
+                          const CUtensorMap& v1, const FwdArgs& args, int BH, cudaStream_t stream);
+
+}  // namespace hmar

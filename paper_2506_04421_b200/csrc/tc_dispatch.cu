@@ -1,15 +1,172 @@
-// Dispatch of the bf16 entry points to the tensor-core kernels, and the per-schedule plan cache.
+// Host-side dispatch of the bf16 entry points to the tensor-core kernels: the per-schedule plan
+// cache (device work lists) and the TMA tensor maps.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <map>
+#include <mutex>
+#include <vector>
+
 #include "launchers.h"
+#include "tc_common.h"
 #include "tc_launchers.h"
 
 namespace hmar {
 
 typedef __nv_bfloat16 bf16;
 
+// ------------------------------------------------------------------------------------------------
+// cuTensorMapEncodeTiled is fetched through the runtime so the library has no link-time dependency
+// on libcuda (it must load on machines without a driver, where only host-side calls are used).
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    });
+    return fn;
+}
+
+// Tensor map of a [heads, rows, 64] bf16 tensor read in boxes of 128 rows x 64 columns with the
+// 128-byte swizzle; rows past the end of a head read as zeros.
+static bool make_rows_map(CUtensorMap* map, const void* base, int heads, int rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows, (cuuint64_t)heads};
+    const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)rows * kHeadDim * 2};
+    const cuuint32_t box[3] = {(cuuint32_t)kHeadDim, (cuuint32_t)kTileRows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Plan cache: one entry per (device, side length list).
+struct Plan {
+    FwdWork* fwd_work = nullptr;
+    int n_fwd = 0;
+};
+
+struct PlanKey {
+    int device;
+    std::vector<int> starts;
+    bool operator<(const PlanKey& o) const {
+        return device != o.device ? device < o.device : starts < o.starts;
+    }
+};
+
+static std::mutex g_plan_mu;
+static std::map<PlanKey, Plan> g_plans;
+
+static const Plan* get_plan(const ScaleTable& st) {
+    PlanKey key;
+    if (cudaGetDevice(&key.device) != cudaSuccess) return nullptr;
+    key.starts.assign(st.start, st.start + st.n_scales + 1);
+    std::lock_guard<std::mutex> lock(g_plan_mu);
+    auto it = g_plans.find(key);
+    if (it != g_plans.end()) return &it->second;
+
+    std::vector<Tile> tiles = build_tiles(st, 0);
+    std::vector<FwdWork> work(tiles.size());
+    for (size_t i = 0; i < tiles.size(); ++i) {
+        work[i].row_begin = tiles[i].row_begin;
+        work[i].row_count = tiles[i].row_count;
+        work[i].s0_begin = tiles[i].partner_begin;
+        work[i].s0_end = tiles[i].partner_end;
+        work[i].s1_begin = work[i].s1_end = 0;
+        work[i].uniform = tiles[i].uniform;
+        work[i].pad = 0;
+    }
+    Plan plan;
+    plan.n_fwd = (int)work.size();
+    cudaStream_t s = nullptr;
+    bool ok = cudaMalloc(&plan.fwd_work, work.size() * sizeof(FwdWork)) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaMemcpyAsync(plan.fwd_work, work.data(), work.size() * sizeof(FwdWork), cudaMemcpyHostToDevice, s) ==
+                  cudaSuccess &&
+              cudaStreamSynchronize(s) == cudaSuccess;
+    if (s != nullptr) cudaStreamDestroy(s);
+    if (!ok) {
+        cudaGetLastError();
+        if (plan.fwd_work) cudaFree(plan.fwd_work);
+        return nullptr;
+    }
+    return &(g_plans[key] = plan);
+}
+
+void tc_release_plans() {
+    std::lock_guard<std::mutex> lock(g_plan_mu);
+    int current = 0;
+    const bool have_dev = cudaGetDevice(&current) == cudaSuccess;
+    for (auto& kv : g_plans) {
+        if (have_dev) cudaSetDevice(kv.first.device);
+        if (kv.second.fwd_work) cudaFree(kv.second.fwd_work);
+    }
+    if (have_dev) cudaSetDevice(current);
+    g_plans.clear();
+    cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
 int tc_fwd(const bf16* q, const bf16* k, const bf16* v, bf16* out, float* lse, int BH, const ScaleTable& st,
            float scale, int* status, cudaStream_t stream) {
-    (void)status;
-    return simt_fwd<bf16>(q, k, v, out, lse, BH, st, scale, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
+    const Plan* plan = get_plan(st);
+    if (plan == nullptr) return HMAR_ERR_CUDA;
+    const int L = st.start[st.n_scales];
+    CUtensorMap mq, mk, mv;
+    if (!make_rows_map(&mq, q, BH, L) || !make_rows_map(&mk, k, BH, L) || !make_rows_map(&mv, v, BH, L))
+        return HMAR_ERR_CUDA;
+    FwdArgs a{};
+    a.work = plan->fwd_work;
+    a.n_work = plan->n_fwd;
+    a.n_q_rows = L;
+    a.n0 = L;
+    a.n1 = 0;
+    a.scale_log2 = scale * 1.4426950408889634f;
+    a.out = out;
+    a.lse = lse;
+    a.status = status;
+    a.st = st;
+    return launch_fwd_tc(mq, mk, mv, mk, mv, a, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
+}
+
+int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const bf16* k_cur, const bf16* v_cur,
+                  bf16* out, float* lse, int BH, int n_prev, int n_cur, float scale, int* status,
+                  cudaStream_t stream) {
+    CUtensorMap mq, mk0, mv0, mk1, mv1;
+    if (!make_rows_map(&mq, q, BH, n_cur) || !make_rows_map(&mk1, k_cur, BH, n_cur) ||
+        !make_rows_map(&mv1, v_cur, BH, n_cur))
+        return HMAR_ERR_CUDA;
+    if (n_prev > 0) {
+        if (!make_rows_map(&mk0, k_prev, BH, n_prev) || !make_rows_map(&mv0, v_prev, BH, n_prev))
+            return HMAR_ERR_CUDA;
+    } else {
+        mk0 = mk1;
+        mv0 = mv1;
+    }
+    FwdArgs a{};
+    a.work = nullptr;
+    a.n_work = (n_cur + kTileRows - 1) / kTileRows;
+    a.n_q_rows = n_cur;
+    a.n0 = n_prev;
+    a.n1 = n_cur;
+    a.scale_log2 = scale * 1.4426950408889634f;
+    a.out = out;
+    a.lse = lse;
+    a.status = status;
+    a.st.n_scales = 0;
+    return launch_fwd_tc(mq, mk0, mv0, mk1, mv1, a, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
 int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const float* lse, const bf16* dout,
@@ -19,15 +176,5 @@ int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const f
     return simt_bwd<bf16>(q, k, v, out, lse, dout, dq, dk, dv, delta, BH, st, scale, stream) == cudaSuccess
                ? HMAR_OK : HMAR_ERR_CUDA;
 }
-
-int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const bf16* k_cur, const bf16* v_cur,
-                  bf16* out, float* lse, int BH, int n_prev, int n_cur, float scale, int* status,
-                  cudaStream_t stream) {
-    (void)status;
-    return simt_scale_step<bf16>(q, k_prev, v_prev, k_cur, v_cur, out, lse, BH, n_prev, n_cur, scale, stream)
-                   == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
-}
-
-void tc_release_plans() {}
 
 }  // namespace hmar
