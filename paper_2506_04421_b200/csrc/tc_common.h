@@ -29,7 +29,34 @@ struct FwdArgs {
     ScaleTable st;
 };
 
+// Backward work tile: key rows [row_begin, row_begin + row_count) and the query range that may see them.
+struct BwdWork {
+    int32_t row_begin, row_count;
+    int32_t q_begin, q_end;
+    int32_t uniform;
+    int32_t pad[3];
+};
+
+struct BwdArgs {
+    const BwdWork* work;
+    int n_work;
+    int L;
+    float scale_log2;        // softmax_scale * log2(e)
+    float softmax_scale;
+    const float* lse;        // [BH, L] from the forward
+    const float* delta;      // [BH, L] rowsum(dO o O) (read by the main kernel)
+    float* delta_w;          // same buffer, written by the preprocess kernel
+    float* dq_acc;           // [BH, L, 64] fp32 accumulator
+    __nv_bfloat16* dk;
+    __nv_bfloat16* dv;
+    int* status;
+    ScaleTable st;
+};
+
 size_t fwd_tc_smem_bytes();
+cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& dout_map,
+                          const BwdArgs& args, const __nv_bfloat16* out, const __nv_bfloat16* dout,
+                          __nv_bfloat16* dq, int BH, cudaStream_t stream);
 cudaError_t launch_fwd_tc(const CUtensorMap& q, const CUtensorMap& k0, const CUtensorMap& v0, const CUtensorMap& k1,
                           const CUtensorMap& v1, const FwdArgs& args, int BH, cudaStream_t stream);
 

@@ -54,8 +54,10 @@ static bool make_rows_map(CUtensorMap* map, const void* base, int heads, int row
 // ------------------------------------------------------------------------------------------------
 // Plan cache: one entry per (device, side length list).
 struct Plan {
-    FwdWork* fwd_work = nullptr;
+    FwdWork* fwd_work = nullptr;     // one allocation: forward tiles, then backward tiles
+    BwdWork* bwd_work = nullptr;
     int n_fwd = 0;
+    int n_bwd = 0;
 };
 
 struct PlanKey {
@@ -88,14 +90,29 @@ static const Plan* get_plan(const ScaleTable& st) {
         work[i].uniform = tiles[i].uniform;
         work[i].pad = 0;
     }
+    std::vector<Tile> btiles = build_tiles(st, 1);
+    std::vector<BwdWork> bwork(btiles.size());
+    for (size_t i = 0; i < btiles.size(); ++i) {
+        bwork[i] = BwdWork{};
+        bwork[i].row_begin = btiles[i].row_begin;
+        bwork[i].row_count = btiles[i].row_count;
+        bwork[i].q_begin = btiles[i].partner_begin;
+        bwork[i].q_end = btiles[i].partner_end;
+        bwork[i].uniform = btiles[i].uniform;
+    }
+    static_assert(sizeof(FwdWork) == sizeof(BwdWork), "work tiles share one allocation");
     Plan plan;
     plan.n_fwd = (int)work.size();
+    plan.n_bwd = (int)bwork.size();
+    const size_t fwd_bytes = work.size() * sizeof(FwdWork), bwd_bytes = bwork.size() * sizeof(BwdWork);
     cudaStream_t s = nullptr;
-    bool ok = cudaMalloc(&plan.fwd_work, work.size() * sizeof(FwdWork)) == cudaSuccess &&
+    bool ok = cudaMalloc(&plan.fwd_work, fwd_bytes + bwd_bytes) == cudaSuccess &&
               cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) == cudaSuccess &&
-              cudaMemcpyAsync(plan.fwd_work, work.data(), work.size() * sizeof(FwdWork), cudaMemcpyHostToDevice, s) ==
-                  cudaSuccess &&
+              cudaMemcpyAsync(plan.fwd_work, work.data(), fwd_bytes, cudaMemcpyHostToDevice, s) == cudaSuccess &&
+              cudaMemcpyAsync(reinterpret_cast<char*>(plan.fwd_work) + fwd_bytes, bwork.data(), bwd_bytes,
+                              cudaMemcpyHostToDevice, s) == cudaSuccess &&
               cudaStreamSynchronize(s) == cudaSuccess;
+    plan.bwd_work = reinterpret_cast<BwdWork*>(reinterpret_cast<char*>(plan.fwd_work) + fwd_bytes);
     if (s != nullptr) cudaStreamDestroy(s);
     if (!ok) {
         cudaGetLastError();
@@ -172,9 +189,28 @@ int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const b
 int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const float* lse, const bf16* dout,
            bf16* dq, bf16* dk, bf16* dv, float* delta, float* dq_acc, int BH, const ScaleTable& st, float scale,
            int* status, cudaStream_t stream) {
-    (void)status; (void)dq_acc;
-    return simt_bwd<bf16>(q, k, v, out, lse, dout, dq, dk, dv, delta, BH, st, scale, stream) == cudaSuccess
-               ? HMAR_OK : HMAR_ERR_CUDA;
+    const Plan* plan = get_plan(st);
+    if (plan == nullptr) return HMAR_ERR_CUDA;
+    const int L = st.start[st.n_scales];
+    CUtensorMap mq, mk, mv, mdo;
+    if (!make_rows_map(&mq, q, BH, L) || !make_rows_map(&mk, k, BH, L) || !make_rows_map(&mv, v, BH, L) ||
+        !make_rows_map(&mdo, dout, BH, L))
+        return HMAR_ERR_CUDA;
+    BwdArgs a{};
+    a.work = plan->bwd_work;
+    a.n_work = plan->n_bwd;
+    a.L = L;
+    a.scale_log2 = scale * 1.4426950408889634f;
+    a.softmax_scale = scale;
+    a.lse = lse;
+    a.delta = delta;
+    a.delta_w = delta;
+    a.dq_acc = dq_acc;
+    a.dk = dk;
+    a.dv = dv;
+    a.status = status;
+    a.st = st;
+    return launch_bwd_tc(mq, mk, mv, mdo, a, out, dout, dq, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
 }  // namespace hmar
