@@ -79,6 +79,29 @@ int hmar_attn_bwd_f32(const float* q, const float* k, const float* v, const floa
                       int B, int H, int D, int n_scales, const int* side_lens,
                       float softmax_scale, void* stream);
 
+/* Backward for callers that cannot allocate device memory (the paper has no counterpart; this is a
+ * library convenience).  Same inputs, outputs and arithmetic as hmar_attn_bwd (bf16), but no workspace
+ * argument and no plan cache: the work list, delta and the fp32 dQ accumulator live in one fixed
+ * device array inside the library image (about 8.6 MB, held by every GPU that loads the library until
+ * the process exits).  It is meant for code that runs where cudaMalloc is off limits: under a framework
+ * that owns all device memory through its own pool, inside a server plug-in that must not grow after
+ * start-up, or wherever a call that may synchronise the device is forbidden.
+ *   - Limit: B * H * L <= HMAR_NOALLOC_MAX_ROWS (and at most 512 work tiles per head); larger problems
+ *     are rejected with HMAR_ERR_WORKSPACE before anything is launched.
+ *   - The call itself never calls cudaMalloc, cudaFree or any allocating routine.  Its first call on a
+ *     device looks up the array's device address (cudaGetSymbolAddress); make that first call outside
+ *     any stream capture.
+ *   - All calls on a device share the array.  The array keeps whatever the previous call left in it;
+ *     each call overwrites the work list and delta and clears the accumulator itself.  Two calls whose
+ *     GPU work may overlap (different streams without an ordering between them) race on it: keep
+ *     calls to this entry point on one stream, or order them with events.
+ *   - Kernel waits that run out are not reported through hmar_device_status() for this entry point. */
+#define HMAR_NOALLOC_MAX_ROWS 32768
+int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                          const void* dout, void* dq, void* dk, void* dv,
+                          int B, int H, int D, int n_scales, const int* side_lens,
+                          float softmax_scale, void* stream);
+
 /* Inference step of one scale (Sec. 4.1: no prefix computation or KV cache beyond the previous
  * scale; Sec. 4.2/4.4: every masked refinement sub-step of scale k sees scale k-1 and scale k).
  *   q            : [B,H,n_cur,D]      queries of the current scale, n_cur = side_cur^2

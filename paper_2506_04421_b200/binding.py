@@ -23,7 +23,7 @@ HMAR_ERR_DEVICE_TIMEOUT = -5
 
 EXPORTED_SYMBOLS = (
     "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd",
-    "hmar_attn_bwd_f32", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_schedule_tiles",
+    "hmar_attn_bwd_f32", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_schedule_tiles",
     "hmar_device_status", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
     "hmar_status_string",
 )
@@ -52,6 +52,7 @@ def lib():
     L.hmar_attn_bwd_workspace_bytes.restype = ctypes.c_size_t
     L.hmar_attn_bwd.argtypes = [vp] * 9 + [vp, ctypes.c_size_t, i, i, i, i, ip, fp, vp]
     L.hmar_attn_bwd_f32.argtypes = L.hmar_attn_bwd.argtypes
+    L.hmar_attn_bwd_noalloc.argtypes = [vp] * 9 + [i, i, i, i, ip, fp, vp]
     L.hmar_attn_scale_step.argtypes = [vp] * 7 + [i, i, i, i, i, fp, vp]
     L.hmar_attn_scale_step_f32.argtypes = L.hmar_attn_scale_step.argtypes
     L.hmar_schedule_tiles.argtypes = [i, ip, i, ctypes.POINTER(ctypes.c_int32), i]
@@ -142,6 +143,25 @@ def hmar_attn_bwd(q, k, v, out, lse, dout, side_lens, softmax_scale, dq=None, dk
     _check(fn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv),
               _ptr(workspace), workspace.numel() * workspace.element_size(), B, H, D, n, sides,
               float(softmax_scale), _stream(stream)), "hmar_attn_bwd")
+    return dq, dk, dv
+
+
+HMAR_NOALLOC_MAX_ROWS = 32768
+
+
+def hmar_attn_bwd_noalloc(q, k, v, out, lse, dout, side_lens, softmax_scale, dq, dk, dv, stream=None):
+    """Backward through the entry point that allocates nothing: for callers that may not touch the
+    device allocator (memory owned by someone else's pool, no growth after start-up, no call that may
+    synchronise). The caller passes every output tensor; neither this wrapper nor the library
+    allocates. B*H*L must not exceed HMAR_NOALLOC_MAX_ROWS, and calls must not overlap on the GPU."""
+    _need(q, k, v, out, lse, dout, dq, dk, dv)
+    if _is_f32(q):
+        raise TypeError("hmar_attn_bwd_noalloc takes bfloat16 tensors")
+    B, H, L, D = q.shape
+    sides, n = _sides(side_lens)
+    _check(lib().hmar_attn_bwd_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), _ptr(dq),
+                                       _ptr(dk), _ptr(dv), B, H, D, n, sides, float(softmax_scale),
+                                       _stream(stream)), "hmar_attn_bwd_noalloc")
     return dq, dk, dv
 
 

@@ -213,4 +213,9 @@ int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const f
     return launch_bwd_tc(mq, mk, mv, mdo, a, out, dout, dq, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
+// Same tensor map as above for code outside this file.
+bool make_rows_map_bf16(CUtensorMap* map, const void* base, int heads, int rows) {
+    return make_rows_map(map, base, heads, rows);
+}
+
 }  // namespace hmar
