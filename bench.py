@@ -191,6 +191,7 @@ def run_ours(args, wl):
         time.sleep(0.3)
     launches0 = hmar.hmar_launch_count()
     barrier()
+    hmar.hmar_profile_begin()          # per-kernel CUDA events on the launch stream, inside the timed region
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     t_begin.record()
@@ -202,6 +203,7 @@ def run_ours(args, wl):
         ev[i][2].record()
     t_end.record()
     barrier()
+    kernels = hmar.hmar_profile_end()
     launches = hmar.hmar_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     total_ms = t_begin.elapsed_time(t_end)
@@ -212,6 +214,8 @@ def run_ours(args, wl):
         raise RuntimeError(f"device status {status} detail {detail:#x}")
 
     # ---- end to end: pinned host tensors in, results back to the host, inside the timed region
+    if args.no_e2e:
+        return _finish(args, wl, world, rank, dev, total_ms, float("nan"), fwd_ms, bwd_ms, launches, clocks, kernels)
     hq, hk, hv, hdo = (t.cpu().pin_memory() for t in (q, k, v, do))
     h_out, h_dq, h_dk, h_dv = (torch.empty_like(hq).pin_memory() for _ in range(4))
     h_lse = torch.empty((B, H, L), dtype=torch.float32).pin_memory()
@@ -238,7 +242,14 @@ def run_ours(args, wl):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    return _finish(args, wl, world, rank, dev, total_ms, e2e_ms, fwd_ms, bwd_ms, launches, clocks, kernels)
 
+
+def _finish(args, wl, world, rank, dev, total_ms, e2e_ms, fwd_ms, bwd_ms, launches, clocks, kernels):
+    import torch
+    import torch.distributed as dist
+    B, H, L, D = wl.B, wl.H, wl.L, wl.D
+    sides, scale = wl.side_lens, wl.softmax_scale
     times = torch.tensor([total_ms, e2e_ms, fwd_ms, bwd_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(times, op=dist.ReduceOp.MAX)
@@ -252,23 +263,30 @@ def run_ours(args, wl):
         peaks = measured_peaks()
         bwd_tf = f_bwd / (bwd_ms * 1e-3) / 1e12
         fwd_tf = f_fwd / (fwd_ms * 1e-3) / 1e12
-        cpu_base, _ = time_oracle(wl, 24, 2, 0)
+        # the dominant kernel: average launch duration from the library's own events in the timed region
+        per_kernel = {name: {"launches": n, "avg_ms": ms / n, "share": ms / (ms_per_step * args.steps)}
+                      for name, (n, ms) in kernels.items()}
+        dom = "hmar_bwd_tc_kernel"
+        dom_ms = per_kernel[dom]["avg_ms"]
+        dom_tf = f_bwd / (dom_ms * 1e-3) / 1e12
+        cpu_base = None if args.no_cpu else time_oracle(wl, min(24, B * H), 2, 0)[0]
         elem = 2 * B * H * L * D
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "B": B, "H": H, "L": L, "D": D, "side_lens": list(sides),
-                       "softmax_scale": scale, "passes": "fwd+bwd", "parallelism": f"replicas x{world}",
+            "config": {"workload": WORKLOAD + (f" (batch reduced to {B})" if args.batch > 0 else ""),
+                       "B": B, "H": H, "L": L, "D": D, "side_lens": list(sides), "softmax_scale": scale, "passes": "fwd+bwd", "parallelism": f"replicas x{world}",
                        "l2": "tensors larger than L2 (8 x 110 MB + 446 MB scratch per step), no flush"},
             "fraction_of_peak": {"burst": value / world / peaks["bf16_tflops"],
                                  "sustained": value / world / (peaks["bf16_tflops_sustained"] or float("nan")),
                                  "nominal_2250": value / world / 2250.0, "peaks": peaks["source"]},
             "phases": {"fwd_ms": fwd_ms, "bwd_ms": bwd_ms, "fwd_tflops": fwd_tf, "bwd_tflops": bwd_tf},
-            "roofline": {"bound": "tensor", "kernel": "backward call (delta + main + dq convert)",
-                         "achieved": bwd_tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                         "frac": bwd_tf / peaks["bf16_tflops"], "peak_source": peaks["source"] + " burst",
-                         "traffic": NCU_TRAFFIC_BYTES["hmar_bwd"]},
+            "roofline": {"bound": "tensor", "kernel": dom, "achieved": dom_tf, "peak": peaks["bf16_tflops"],
+                         "unit": "TFLOP/s", "frac": dom_tf / peaks["bf16_tflops"],
+                         "peak_source": peaks["source"] + " burst", "avg_launch_ms": dom_ms,
+                         "algorithmic_flops_per_launch": f_bwd, "traffic": NCU_TRAFFIC_BYTES["hmar_bwd"]},
+            "kernels": per_kernel,
             "cpu_baseline": cpu_base,
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": 4 * elem, "d2h_bytes_per_step": 4 * elem + 4 * B * H * L},
@@ -286,10 +304,17 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--batch", type=int, default=0,
+                    help="override the batch size (profiling on a reduced case; named in config.workload)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from workloads import CONFIGS
     wl = CONFIGS[WORKLOAD]
+    if args.batch > 0:
+        import dataclasses
+        wl = dataclasses.replace(wl, B=args.batch)
     if args.impl == "reference":
         run_reference(args, wl)
     else:

@@ -134,6 +134,13 @@ int hmar_schedule_tiles(int n_scales, const int* side_lens, int direction,
  * telling which wait gave up) and clears it.  Diagnostics only; never needed for correct results. */
 int hmar_device_status(int* detail);
 
+/* Per-kernel timing for benchmarks.  Between hmar_profile_begin() and hmar_profile_end() every kernel
+ * the library launches is bracketed by two CUDA events on its stream.  hmar_profile_end() synchronises
+ * the device and writes one line per kernel name, "name launches total_ms\n", into `report`
+ * (NUL-terminated, truncated to `capacity`).  Not thread-safe against concurrent entry-point calls. */
+void hmar_profile_begin(void);
+int hmar_profile_end(char* report, size_t capacity);
+
 /* Debug switch: nonzero routes the bf16 entry points through the plain SIMT kernels (the same ones
  * the _f32 build uses) instead of the tensor-core kernels.  Returns the previous setting. */
 int hmar_debug_force_simt(int enable);

@@ -24,7 +24,7 @@ HMAR_ERR_DEVICE_TIMEOUT = -5
 EXPORTED_SYMBOLS = (
     "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd",
     "hmar_attn_bwd_f32", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_schedule_tiles",
-    "hmar_device_status", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
+    "hmar_device_status", "hmar_profile_begin", "hmar_profile_end", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
     "hmar_status_string",
 )
 
@@ -57,6 +57,8 @@ def lib():
     L.hmar_attn_scale_step_f32.argtypes = L.hmar_attn_scale_step.argtypes
     L.hmar_schedule_tiles.argtypes = [i, ip, i, ctypes.POINTER(ctypes.c_int32), i]
     L.hmar_device_status.argtypes = [ip]
+    L.hmar_profile_begin.restype = None
+    L.hmar_profile_end.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
     L.hmar_debug_force_simt.argtypes = [i]
     L.hmar_launch_count.restype = ctypes.c_longlong
     L.hmar_shutdown.restype = None
@@ -199,6 +201,21 @@ def hmar_device_status():
     detail = ctypes.c_int(0)
     status = lib().hmar_device_status(ctypes.byref(detail))
     return status, detail.value
+
+
+def hmar_profile_begin():
+    lib().hmar_profile_begin()
+
+
+def hmar_profile_end():
+    """{kernel name: (launches, total_ms)} for the kernels launched since hmar_profile_begin()."""
+    buf = ctypes.create_string_buffer(8192)
+    _check(lib().hmar_profile_end(buf, len(buf)), "hmar_profile_end")
+    out = {}
+    for line in buf.value.decode().splitlines():
+        name, count, ms = line.split()
+        out[name] = (int(count), float(ms))
+    return out
 
 
 def hmar_debug_force_simt(enable):

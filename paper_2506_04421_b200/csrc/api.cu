@@ -3,9 +3,11 @@
 #include <cuda_runtime.h>
 
 #include <atomic>
+#include <cstdio>
 #include <cstring>
 #include <map>
 #include <mutex>
+#include <string>
 #include <type_traits>
 #include <vector>
 
@@ -18,6 +20,33 @@ namespace hmar {
 static std::atomic<long long> g_launches{0};
 static std::atomic<int> g_force_simt{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// ---- per-kernel timing
+struct TimedLaunch { const char* name; cudaEvent_t begin, end; };
+static std::atomic<int> g_profile_on{0};
+static std::mutex g_profile_mu;
+static std::vector<TimedLaunch> g_profile_log;
+
+bool profile_enabled() { return g_profile_on.load(std::memory_order_relaxed) != 0; }
+
+KernelTimer::KernelTimer(const char* name, cudaStream_t stream)
+    : name_(name), stream_(stream), begin_(nullptr), on_(profile_enabled()) {
+    if (on_ && (cudaEventCreate(&begin_) != cudaSuccess || cudaEventRecord(begin_, stream_) != cudaSuccess)) {
+        cudaGetLastError();
+        on_ = false;
+    }
+}
+
+KernelTimer::~KernelTimer() {
+    if (!on_) return;
+    cudaEvent_t end = nullptr;
+    if (cudaEventCreate(&end) == cudaSuccess && cudaEventRecord(end, stream_) == cudaSuccess) {
+        std::lock_guard<std::mutex> lock(g_profile_mu);
+        g_profile_log.push_back(TimedLaunch{name_, begin_, end});
+    } else {
+        cudaGetLastError();
+    }
+}
 
 // Device status word written by kernels whose bounded waits ran out: {code, detail}.
 __device__ int g_device_status[2];
@@ -228,6 +257,45 @@ int hmar_device_status(int* detail) {
     if (cudaMemcpyToSymbol(g_device_status, zero, sizeof(zero)) != cudaSuccess) { cudaGetLastError(); return HMAR_ERR_CUDA; }
     if (detail) *detail = host[1];
     return host[0] == 0 ? HMAR_OK : HMAR_ERR_DEVICE_TIMEOUT;
+}
+
+void hmar_profile_begin(void) {
+    std::lock_guard<std::mutex> lock(g_profile_mu);
+    for (auto& t : g_profile_log) { cudaEventDestroy(t.begin); cudaEventDestroy(t.end); }
+    g_profile_log.clear();
+    g_profile_on.store(1);
+}
+
+int hmar_profile_end(char* report, size_t capacity) {
+    g_profile_on.store(0);
+    if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return HMAR_ERR_CUDA; }
+    std::lock_guard<std::mutex> lock(g_profile_mu);
+    std::map<std::string, std::pair<int, double>> acc;
+    for (auto& t : g_profile_log) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, t.begin, t.end) == cudaSuccess) {
+            auto& a = acc[t.name];
+            a.first += 1;
+            a.second += ms;
+        } else {
+            cudaGetLastError();
+        }
+        cudaEventDestroy(t.begin);
+        cudaEventDestroy(t.end);
+    }
+    g_profile_log.clear();
+    std::string text;
+    for (auto& kv : acc) {
+        char line[160];
+        snprintf(line, sizeof(line), "%s %d %.6f\n", kv.first.c_str(), kv.second.first, kv.second.second);
+        text += line;
+    }
+    if (report != nullptr && capacity > 0) {
+        const size_t n = text.size() < capacity - 1 ? text.size() : capacity - 1;
+        std::memcpy(report, text.data(), n);
+        report[n] = 0;
+    }
+    return HMAR_OK;
 }
 
 int hmar_debug_force_simt(int enable) { return g_force_simt.exchange(enable ? 1 : 0); }

@@ -390,12 +390,24 @@ cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUte
     cudaError_t e = cudaFuncSetAttribute(hmar_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const size_t n_rows = (size_t)BH * args.L;
-    e = cudaMemsetAsync(args.dq_acc, 0, n_rows * D * sizeof(float), stream);
-    if (e != cudaSuccess) return e;
-    hmar_bwd_delta_kernel<<<(unsigned)((n_rows * 8 + 255) / 256), 256, 0, stream>>>(out, dout, args.delta_w, n_rows);
-    hmar_bwd_tc_kernel<<<(unsigned)BH * (unsigned)args.n_work, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, args);
+    {
+        KernelTimer timer("memset_dq_acc", stream);
+        e = cudaMemsetAsync(args.dq_acc, 0, n_rows * D * sizeof(float), stream);
+        if (e != cudaSuccess) return e;
+    }
+    {
+        KernelTimer timer("hmar_bwd_delta_kernel", stream);
+        hmar_bwd_delta_kernel<<<(unsigned)((n_rows * 8 + 255) / 256), 256, 0, stream>>>(out, dout, args.delta_w, n_rows);
+    }
+    {
+        KernelTimer timer("hmar_bwd_tc_kernel", stream);
+        hmar_bwd_tc_kernel<<<(unsigned)BH * (unsigned)args.n_work, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, args);
+    }
     const size_t n8 = n_rows * D / 8;
-    hmar_bwd_dq_convert_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, stream>>>(args.dq_acc, dq, args.softmax_scale, n8);
+    {
+        KernelTimer timer("hmar_bwd_dq_convert_kernel", stream);
+        hmar_bwd_dq_convert_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, stream>>>(args.dq_acc, dq, args.softmax_scale, n8);
+    }
     count_launch(3);
     return cudaGetLastError();
 }

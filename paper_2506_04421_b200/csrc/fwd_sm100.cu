@@ -358,7 +358,10 @@ cudaError_t launch_fwd_tc(const CUtensorMap& q, const CUtensorMap& k0, const CUt
     cudaError_t e = cudaFuncSetAttribute(hmar_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const unsigned grid = (unsigned)BH * (unsigned)args.n_work;
-    hmar_fwd_tc_kernel<<<grid, NUM_THREADS, smem, stream>>>(q, k0, v0, k1, v1, args);
+    {
+        KernelTimer timer(args.work != nullptr ? "hmar_fwd_tc_kernel" : "hmar_fwd_tc_kernel/scale_step", stream);
+        hmar_fwd_tc_kernel<<<grid, NUM_THREADS, smem, stream>>>(q, k0, v0, k1, v1, args);
+    }
     count_launch(1);
     return cudaGetLastError();
 }

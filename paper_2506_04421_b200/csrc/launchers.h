@@ -7,6 +7,18 @@ namespace hmar {
 
 void count_launch(int n);
 
+// Per-kernel timing (diagnostics): when profiling is on, a kernel launch wrapped in KernelTimer is
+// bracketed by two events on its stream; hmar_profile_end() sums them per kernel name.
+bool profile_enabled();
+struct KernelTimer {
+    KernelTimer(const char* name, cudaStream_t stream);
+    ~KernelTimer();
+    const char* name_;
+    cudaStream_t stream_;
+    cudaEvent_t begin_;
+    bool on_;
+};
+
 template <typename T>
 cudaError_t simt_fwd(const T* q, const T* k, const T* v, T* out, float* lse, int BH,
                      const ScaleTable& st, float scale, cudaStream_t stream);
