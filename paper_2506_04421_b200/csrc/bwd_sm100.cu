@@ -8,8 +8,9 @@
 // Main kernel: one block owns one tile of up to 128 key rows of one head and walks over the
 // contiguous range of query rows that may see them under the mask (queries of the keys' own scale and
 // of the next scale; paper Sec. 4.1, Fig. attn-mask), 128 queries at a time:
-//   warp 8      TMA producer: K, V once; then Q_i, dO_i through a 2-stage ring; lse_i, delta_i by
-//               plain loads (their row offsets are not 16-byte aligned)
+//   warp 8      TMA producer: K, V once; then Q_i, dO_i through a 3-stage ring
+//   warp 10     loads lse_i, delta_i with plain loads (their row offsets are not 16-byte aligned) into
+//               an 8-deep ring
 //   warp 9      issues tcgen05.mma: S^T = K Q_i^T and dP^T = V dO_i^T into TMEM; after the compute
 //               warps are done: dV += P^T dO_i (P^T read from TMEM), dK += dS^T Q_i and
 //               dQ_i = dS K (dS read from shared memory, once as a K-major and once as an
@@ -37,11 +38,12 @@ using namespace ptx;
 constexpr int BKV = 128;             // key rows per block
 constexpr int BQ = 128;              // query rows per step
 constexpr int D = kHeadDim;
-constexpr int NSTAGE = 2;
+constexpr int NSTAGE = 3;
+constexpr int AUX_STAGES = 8;        // ring of lse / delta rows, loaded this many steps ahead
 constexpr int TILE_BYTES = 128 * D * 2;          // 16 KB
 constexpr int NUM_COMPUTE_WARPS = 8;
-constexpr int PRODUCER_WARP = 8, MMA_WARP = 9;
-constexpr int NUM_THREADS = 320;
+constexpr int PRODUCER_WARP = 8, MMA_WARP = 9, AUX_WARP = 10;
+constexpr int NUM_THREADS = 352;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t COL_ST = 0, COL_DPT = 128, COL_DK = 256, COL_DV = 320, COL_DQ = 384;
 
@@ -50,12 +52,12 @@ struct __align__(1024) SharedStorage {
     uint8_t v[TILE_BYTES];
     uint8_t q[NSTAGE][TILE_BYTES];
     uint8_t dout[NSTAGE][TILE_BYTES];
-    uint8_t ds[2][TILE_BYTES];              // dS^T as [64-query block][key row][64 queries], 128B swizzle
-    float lse2[NSTAGE][BQ];                 // lse * log2(e); +inf for query rows outside the range
-    float delta[NSTAGE][BQ];
+    uint8_t ds[2][2][TILE_BYTES];           // dS^T, double buffered: [step parity][64-query half][key row][64 queries], 128B swizzle
+    float lse2[AUX_STAGES][BQ];             // lse * log2(e); +inf for query rows outside the range
+    float delta[AUX_STAGES][BQ];
     uint64_t kv_full;
-    uint64_t qdo_full[NSTAGE], aux_full[NSTAGE], q_empty[NSTAGE];
-    uint64_t s_full, p_full, dq_full;
+    uint64_t qdo_full[NSTAGE], q_empty[NSTAGE], aux_full[AUX_STAGES], aux_empty[AUX_STAGES];
+    uint64_t s_full[2], p_full[2], dq_full;   // [half of the step]
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -72,6 +74,18 @@ __device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float 
                  "f"(d)
                  : "memory");
 }
+
+#ifdef HMAR_STAMPS
+// Developer build only: per-phase clock totals of compute warp 0 and of the MMA thread, summed over blocks.
+__device__ unsigned long long g_bwd_stamps[16];
+#define STAMP_DECL unsigned long long st_acc[16] = {0}; long long st_t = clock64();
+#define STAMP(idx) { long long st_n = clock64(); st_acc[idx] += (unsigned long long)(st_n - st_t); st_t = st_n; }
+#define STAMP_FLUSH(lo, hi) { for (int st_i = lo; st_i < hi; ++st_i) atomicAdd(&g_bwd_stamps[st_i], st_acc[st_i]); }
+#else
+#define STAMP_DECL
+#define STAMP(idx) {}
+#define STAMP_FLUSH(lo, hi) {}
+#endif
 
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -99,11 +113,16 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         mbar_init(&sm.kv_full, 1);
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(&sm.qdo_full[s], 1);
-            mbar_init(&sm.aux_full[s], 32);
             mbar_init(&sm.q_empty[s], 1);
         }
-        mbar_init(&sm.s_full, 1);
-        mbar_init(&sm.p_full, NUM_COMPUTE_WARPS * 32);
+        for (int s = 0; s < AUX_STAGES; ++s) {
+            mbar_init(&sm.aux_full[s], 32);
+            mbar_init(&sm.aux_empty[s], NUM_COMPUTE_WARPS * 32);
+        }
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(&sm.s_full[h], 1);
+            mbar_init(&sm.p_full[h], NUM_COMPUTE_WARPS * 32);
+        }
         mbar_init(&sm.dq_full, 1);
         fence_mbar_init();
     }
@@ -129,96 +148,170 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             tma_load_3d(sm.v, &map_v, &sm.kv_full, 0, w.row_begin, bh);
         }
         bool ok = true;
-        for (int i = 0; i < n_steps; ++i) {
-            const int slot = i % NSTAGE;
-            const int q0 = w.q_begin + i * BQ;
-            if (i >= NSTAGE) {
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_empty[slot], ((i / NSTAGE) & 1) ^ 1, abort_flag));
-                if (!ok) { if (lane == 0) report_timeout(args.status, 0x1100 + i); break; }
-            }
-            if (lane == 0) {
+        if (lane == 0) {
+            for (int i = 0; i < n_steps; ++i) {
+                const int slot = i % NSTAGE;
+                const int q0 = w.q_begin + i * BQ;
+                if (i >= NSTAGE) {
+                    ok = mbar_wait(&sm.q_empty[slot], ((i / NSTAGE) & 1) ^ 1, abort_flag);
+                    if (!ok) { report_timeout(args.status, 0x1100 + i); break; }
+                }
                 mbar_arrive_expect_tx(&sm.qdo_full[slot], 2 * TILE_BYTES);
                 tma_load_3d(sm.q[slot], &map_q, &sm.qdo_full[slot], 0, q0, bh);
                 tma_load_3d(sm.dout[slot], &map_do, &sm.qdo_full[slot], 0, q0, bh);
             }
-#pragma unroll
-            for (int t = 0; t < BQ / 32; ++t) {
-                const int c = t * 32 + lane;
-                const int row = q0 + c;
-                const bool in = row < w.q_end;
-                sm.lse2[slot][c] = in ? args.lse[(size_t)bh * L + row] * 1.4426950408889634f : INFINITY;
-                sm.delta[slot][c] = in ? args.delta[(size_t)bh * L + row] : 0.f;
-            }
-            mbar_arrive(&sm.aux_full[slot]);
         }
         if (!ok && lane == 0) {
             const uint64_t t0 = globaltimer_ns();
             while (globaltimer_ns() - t0 < 2000000ull) { }
         }
+    } else if (warp == AUX_WARP) {
+        // ================================================================== lse / delta loader
+        // lse and delta rows of step i go to ring slot i % AUX_STAGES, several steps ahead of their use
+        // (plain loads: their row offsets are not 16-byte aligned, so TMA cannot fetch them).
+        STAMP_DECL
+        for (int i = 0; i < n_steps; ++i) {
+            const int aslot = i % AUX_STAGES;
+            STAMP(13)
+            if (i >= AUX_STAGES) {
+                const bool ok = __all_sync(0xffffffffu,
+                                           mbar_wait(&sm.aux_empty[aslot], ((i / AUX_STAGES) & 1) ^ 1, abort_flag));
+                if (!ok) { if (lane == 0) report_timeout(args.status, 0x1700 + i); break; }
+            }
+            STAMP(12)
+            const int q0 = w.q_begin + i * BQ;
+            // all loads first, then the stores: stores to shared memory in between would serialise them
+            float lv[BQ / 32], dv[BQ / 32];
+#pragma unroll
+            for (int t = 0; t < BQ / 32; ++t) {
+                const int row = q0 + t * 32 + lane;
+                const bool in = row < w.q_end;
+                lv[t] = in ? __ldg(args.lse + (size_t)bh * L + row) : INFINITY;
+                dv[t] = in ? __ldg(args.delta + (size_t)bh * L + row) : 0.f;
+            }
+#pragma unroll
+            for (int t = 0; t < BQ / 32; ++t) {
+                sm.lse2[aslot][t * 32 + lane] = lv[t] * 1.4426950408889634f;
+                sm.delta[aslot][t * 32 + lane] = dv[t];
+            }
+            mbar_arrive(&sm.aux_full[aslot]);
+        }
+        STAMP(13)
+        if (lane == 0) STAMP_FLUSH(12, 14)
     } else if (warp == MMA_WARP) {
         // ================================================================== MMA issuer
-        if (lane == 0) {
-            const uint32_t k_addr = smem_u32(sm.k), v_addr = smem_u32(sm.v);
-            const uint32_t ds_addr = smem_u32(sm.ds[0]);
-            bool ok = mbar_wait(&sm.kv_full, 0, abort_flag);
-            if (!ok) report_timeout(args.status, 0x1200);
+        // A step of 128 queries is split into two halves of 64 (a: queries 0-63, b: 64-127), each with
+        // its own S^T / dP^T columns and barriers, so that the compute warps work on one half while
+        // the tensor core produces the scores of the other half or consumes the finished one.
+        // The whole warp runs the control flow; one elected lane issues.  Descriptors are built once and
+        // advanced by adding (byte offset >> 4) to them, so issuing an MMA costs a few instructions.
+        {
+            const bool leader = elect_one();
+            STAMP_DECL
+            bool ok = __all_sync(0xffffffffu, mbar_wait(&sm.kv_full, 0, abort_flag));
+            if (!ok && lane == 0) report_timeout(args.status, 0x1200);
+            STAMP(8)
+            const uint64_t k_kd = smem_desc_sw128(smem_u32(sm.k), 16);          // K rows, K-major (A of S^T)
+            const uint64_t v_kd = smem_desc_sw128(smem_u32(sm.v), 16);          // V rows, K-major (A of dP^T)
+            const uint64_t k_mn = smem_desc_sw128(smem_u32(sm.k), 1024);        // K as MN-major B of dQ
+            // the ring slots and the dS buffers are 16 KB apart: descriptor of slot s = base + s * 1024
+            const uint64_t q_kd0 = smem_desc_sw128(smem_u32(sm.q[0]), 16), do_kd0 = smem_desc_sw128(smem_u32(sm.dout[0]), 16);
+            const uint64_t q_mn0 = smem_desc_sw128(smem_u32(sm.q[0]), 1024), do_mn0 = smem_desc_sw128(smem_u32(sm.dout[0]), 1024);
+            const uint64_t ds_kd0 = smem_desc_sw128(smem_u32(sm.ds[0][0]), 16);
+            const uint64_t ds_mn0 = smem_desc_sw128(smem_u32(sm.ds[0][0]), TILE_BYTES);
+            constexpr uint32_t idesc_acc = idesc_bf16_f32(BKV, D, false, true);    // A K-major / TMEM, B MN-major
+            constexpr uint32_t idesc_dq = idesc_bf16_f32(BQ, D, true, true);
 
-            auto n_eff_of = [&](int i) {
+            auto n_eff_half = [&](int i, int h) {
                 const int n_valid = min(BQ, w.q_end - (w.q_begin + i * BQ));
-                return (n_valid + 15) & ~15;
+                const int n_eff = (n_valid + 15) & ~15;
+                return h == 0 ? min(n_eff, 64) : max(n_eff - 64, 0);
             };
-            auto issue_scores = [&](int i) -> bool {     // S^T_i = K Q_i^T,  dP^T_i = V dO_i^T
+            // S^T_h = K Q_h^T,  dP^T_h = V dO_h^T  for half h of step i
+            auto issue_scores = [&](int i, int h) -> bool {
                 const int slot = i % NSTAGE;
-                if (!mbar_wait(&sm.qdo_full[slot], (i / NSTAGE) & 1, abort_flag)) {
-                    report_timeout(args.status, 0x1300 + i);
+                const int n = n_eff_half(i, h);
+                if (n == 0) return true;
+                STAMP(11)
+                if (!__all_sync(0xffffffffu, mbar_wait(&sm.qdo_full[slot], (i / NSTAGE) & 1, abort_flag))) {
+                    if (lane == 0) report_timeout(args.status, 0x1300 + i);
                     return false;
                 }
+                STAMP(9)
                 tc_fence_after();
-                const uint32_t idesc = idesc_bf16_f32(BKV, n_eff_of(i), false, false);
-                const uint32_t q_addr = smem_u32(sm.q[slot]), do_addr = smem_u32(sm.dout[slot]);
+                if (leader) {
+                    const uint32_t idesc = idesc_bf16_f32(BKV, n, false, false);
+                    const uint64_t qd = q_kd0 + slot * 1024 + h * 512, dd = do_kd0 + slot * 1024 + h * 512;
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(tmem + COL_ST, smem_desc_sw128(k_addr + ks * 32, 16), smem_desc_sw128(q_addr + ks * 32, 16),
-                           idesc, ks > 0);
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        mma_ss(tmem + COL_ST + h * 64, k_kd + ks * 2, qd + ks * 2, idesc, ks > 0);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(tmem + COL_DPT, smem_desc_sw128(v_addr + ks * 32, 16),
-                           smem_desc_sw128(do_addr + ks * 32, 16), idesc, ks > 0);
-                tc_commit(&sm.s_full);
+                    for (int ks = 0; ks < D / 16; ++ks)
+                        mma_ss(tmem + COL_DPT + h * 64, v_kd + ks * 2, dd + ks * 2, idesc, ks > 0);
+                    tc_commit(&sm.s_full[h]);
+                }
+                __syncwarp();
+                return true;
+            };
+            // dV += P_h^T dO_h,  dK += dS_h^T Q_h  for half h of step i
+            auto issue_grads = [&](int i, int h) -> bool {
+                const int slot = i % NSTAGE;
+                const int n = n_eff_half(i, h);
+                if (n == 0) return true;
+                STAMP(11)
+                if (!__all_sync(0xffffffffu, mbar_wait(&sm.p_full[h], i & 1, abort_flag))) {
+                    if (lane == 0) report_timeout(args.status, 0x1400 + i);
+                    return false;
+                }
+                STAMP(10)
+                tc_fence_after();
+                if (leader) {
+                    const int nk = n / 16;
+                    const uint64_t dod = do_mn0 + slot * 1024 + h * 512, qd = q_mn0 + slot * 1024 + h * 512;
+                    const uint64_t dsd = ds_kd0 + ((i & 1) * 2 + h) * 1024;
+                    const uint32_t p_base = tmem + COL_ST + h * 64;
+                    const bool first = (i == 0) && (h == 0);
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        if (ks < nk)
+                            mma_ts(tmem + COL_DV, p_base + (ks / 2) * 32 + (ks % 2) * 8, dod + ks * 128, idesc_acc,
+                                   !first || (ks > 0));
+#pragma unroll
+                    for (int ks = 0; ks < 4; ++ks)
+                        if (ks < nk)
+                            mma_ss(tmem + COL_DK, dsd + ks * 2, qd + ks * 128, idesc_acc, !first || (ks > 0));
+                }
+                __syncwarp();
                 return true;
             };
 
-            if (ok) ok = issue_scores(0);
+            if (ok) ok = issue_scores(0, 0);
+            if (ok) ok = issue_scores(0, 1);
             for (int i = 0; i < n_steps && ok; ++i) {
-                const int slot = i % NSTAGE;
-                const int n_eff = n_eff_of(i);
-                ok = mbar_wait(&sm.p_full, i & 1, abort_flag);
-                if (!ok) { report_timeout(args.status, 0x1400 + i); break; }
-                tc_fence_after();
-                const uint32_t q_addr = smem_u32(sm.q[slot]), do_addr = smem_u32(sm.dout[slot]);
-                const uint32_t idesc_acc = idesc_bf16_f32(BKV, D, false, true);    // A K-major / TMEM, B MN-major
-                // dV += P^T dO_i : contraction over the queries of the step
-                for (int ks = 0; ks < n_eff / 16; ++ks)
-                    mma_ts(tmem + COL_DV, tmem + COL_ST + (ks / 4) * 64 + (ks % 4) * 8,
-                           smem_desc_sw128(do_addr + ks * 2048, 1024), idesc_acc, (i > 0) || (ks > 0));
-                // dK += dS^T Q_i : A = dS^T rows (keys) x queries, K-major inside each 64-query block
-                for (int ks = 0; ks < n_eff / 16; ++ks)
-                    mma_ss(tmem + COL_DK, smem_desc_sw128(ds_addr + (ks / 4) * TILE_BYTES + (ks % 4) * 32, 16),
-                           smem_desc_sw128(q_addr + ks * 2048, 1024), idesc_acc, (i > 0) || (ks > 0));
-                // dQ_i = dS K : A = dS (queries x keys) read from the same buffer as an MN-major operand
-                const uint32_t idesc_dq = idesc_bf16_f32(BQ, D, true, true);
-                for (int ks = 0; ks < BKV / 16; ++ks)
-                    mma_ss(tmem + COL_DQ, smem_desc_sw128(ds_addr + ks * 2048, TILE_BYTES),
-                           smem_desc_sw128(k_addr + ks * 2048, 1024), idesc_dq, ks > 0);
-                tc_commit(&sm.q_empty[slot]);
-                tc_commit(&sm.dq_full);
-                if (i + 1 < n_steps) ok = issue_scores(i + 1);
+                ok = issue_grads(i, 0);
+                if (ok && i + 1 < n_steps) ok = issue_scores(i + 1, 0);
+                if (ok) ok = issue_grads(i, 1);
+                if (!ok) break;
+                // dQ_i = dS K over both halves: A = dS (queries x keys) read as an MN-major operand.  When
+                // the step has no second half its rows are stale data and are never drained.
+                if (leader) {
+                    const uint64_t dsd = ds_mn0 + (i & 1) * 2048;
+#pragma unroll
+                    for (int ks = 0; ks < BKV / 16; ++ks)
+                        mma_ss(tmem + COL_DQ, dsd + ks * 128, k_mn + ks * 128, idesc_dq, ks > 0);
+                    tc_commit(&sm.q_empty[i % NSTAGE]);
+                    tc_commit(&sm.dq_full);
+                }
+                __syncwarp();
+                if (i + 1 < n_steps) ok = issue_scores(i + 1, 1);
             }
+            STAMP(11)
+            if (lane == 0) STAMP_FLUSH(8, 12)
         }
     } else {
         // ================================================================== compute warps
         const int quarter = warp & 3;
-        const int half = warp >> 2;                         // which 64 query columns of the step
+        const int grp = warp >> 2;                          // which 32 query columns of a half
         const int j = quarter * 32 + lane;                  // key row inside the tile
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
         const bool row_ok = j < w.row_count;
@@ -230,81 +323,121 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
         const bool tile_masked = (!w.uniform) || (w.row_count < BKV);
         const float sl2 = args.scale_log2;
-        uint8_t* ds_row = sm.ds[half] + (j >> 3) * 1024 + (j & 7) * 128;
+        const int ds_row_off = (j >> 3) * 1024 + (j & 7) * 128;
         bool ok = true;
         uint32_t s_buf[32], dp_buf[32];
+        STAMP_DECL
 
-        for (int i = 0; i < n_steps; ++i) {
+        // drains dQ of step `i` from TMEM into the fp32 accumulator (this thread: one query row, 32 dims)
+        auto drain_dq = [&](int i) -> bool {
+            if (!__all_sync(0xffffffffu, mbar_wait(&sm.dq_full, i & 1, abort_flag))) {
+                if (lane == 0) report_timeout(args.status, 0x1600 + i);
+                return false;
+            }
+            STAMP(3)
+            tc_fence_after();
+            const int q0 = w.q_begin + i * BQ;
+            const int n_valid = min(BQ, w.q_end - q0);
+            tmem_ld32(lane_base + COL_DQ + grp * 32, s_buf);
+            tmem_ld_wait();
+            if (j < n_valid) {
+                float* dst = args.dq_acc + ((size_t)bh * L + q0 + j) * D + grp * 32;
+#pragma unroll
+                for (int t = 0; t < 32; t += 4)
+                    red_add_v4(dst + t, __uint_as_float(s_buf[t]), __uint_as_float(s_buf[t + 1]),
+                               __uint_as_float(s_buf[t + 2]), __uint_as_float(s_buf[t + 3]));
+            }
+            tc_fence_before();
+            STAMP(4)
+            return true;
+        };
+
+        for (int i = 0; i < n_steps && ok; ++i) {
             const int slot = i % NSTAGE;
             const int q0 = w.q_begin + i * BQ;
             const int n_valid = min(BQ, w.q_end - q0);
             const int n_eff = (n_valid + 15) & ~15;
-
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.aux_full[slot], (i / NSTAGE) & 1, abort_flag));
-            if (ok) ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full, i & 1, abort_flag));
-            if (!ok) { if (lane == 0) report_timeout(args.status, 0x1500 + i); break; }
-            tc_fence_after();
-
             // visible query columns of this key row in this step: [c_lo, c_hi)
             const int c_lo = row_ok ? max(qlo - q0, 0) : 0;
             const int c_hi = row_ok ? min(qhi - q0, n_valid) : 0;
 
-#pragma unroll
-            for (int cc = 0; cc < 2; ++cc) {
-                const int c0 = half * 64 + cc * 32;
+            const int aslot = i % AUX_STAGES;
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.aux_full[aslot], (i / AUX_STAGES) & 1, abort_flag));
+            if (!ok) { if (lane == 0) report_timeout(args.status, 0x1500 + i); break; }
+#ifdef HMAR_STAMPS
+            if (i == 0) STAMP(6) else STAMP(0)
+#endif
+
+            // dQ of the previous step must leave TMEM before this step's dQ is issued, i.e. before the
+            // last arrival of this step.  With two halves it is drained between them (the tensor core
+            // has finished it by then); a step with a single half drains it first.
+            const bool has_b = n_eff > 64;
+            if (i > 0 && !has_b) ok = drain_dq(i - 1);
+
+            for (int h = 0; h < 2 && ok; ++h) {
+                if (h == 1 && !has_b) break;
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[h], i & 1, abort_flag));
+                if (!ok) { if (lane == 0) report_timeout(args.status, 0x1580 + i); break; }
+                STAMP(1)
+                tc_fence_after();
+                const int c0 = h * 64 + grp * 32;           // first query column of this thread's chunk
                 if (c0 < n_eff) {
                     tmem_ld32(lane_base + COL_ST + c0, s_buf);
                     tmem_ld32(lane_base + COL_DPT + c0, dp_buf);
+                    // lse / delta of the chunk's 32 queries while the TMEM loads are in flight
+                    float4 ls[8], de[8];
+                    const float4* lse4 = reinterpret_cast<const float4*>(&sm.lse2[aslot][c0]);
+                    const float4* del4 = reinterpret_cast<const float4*>(&sm.delta[aslot][c0]);
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) { ls[t] = lse4[t]; de[t] = del4[t]; }
                     tmem_ld_wait();
+                    STAMP(14)
                     uint32_t p_pack[16], ds_pack[16];
 #pragma unroll
-                    for (int t = 0; t < 32; t += 2) {
-                        const float l0 = sm.lse2[slot][c0 + t], l1 = sm.lse2[slot][c0 + t + 1];
-                        float p0 = ex2(fmaf(__uint_as_float(s_buf[t]), sl2, -l0));
-                        float p1 = ex2(fmaf(__uint_as_float(s_buf[t + 1]), sl2, -l1));
+                    for (int t = 0; t < 32; t += 4) {
+                        float p0 = ex2(fmaf(__uint_as_float(s_buf[t]), sl2, -ls[t / 4].x));
+                        float p1 = ex2(fmaf(__uint_as_float(s_buf[t + 1]), sl2, -ls[t / 4].y));
+                        float p2 = ex2(fmaf(__uint_as_float(s_buf[t + 2]), sl2, -ls[t / 4].z));
+                        float p3 = ex2(fmaf(__uint_as_float(s_buf[t + 3]), sl2, -ls[t / 4].w));
                         if (tile_masked) {
                             p0 = (c0 + t >= c_lo && c0 + t < c_hi) ? p0 : 0.f;
                             p1 = (c0 + t + 1 >= c_lo && c0 + t + 1 < c_hi) ? p1 : 0.f;
+                            p2 = (c0 + t + 2 >= c_lo && c0 + t + 2 < c_hi) ? p2 : 0.f;
+                            p3 = (c0 + t + 3 >= c_lo && c0 + t + 3 < c_hi) ? p3 : 0.f;
                         }
-                        const float d0 = p0 * (__uint_as_float(dp_buf[t]) - sm.delta[slot][c0 + t]);
-                        const float d1 = p1 * (__uint_as_float(dp_buf[t + 1]) - sm.delta[slot][c0 + t + 1]);
+                        const float d0 = p0 * (__uint_as_float(dp_buf[t]) - de[t / 4].x);
+                        const float d1 = p1 * (__uint_as_float(dp_buf[t + 1]) - de[t / 4].y);
+                        const float d2 = p2 * (__uint_as_float(dp_buf[t + 2]) - de[t / 4].z);
+                        const float d3 = p3 * (__uint_as_float(dp_buf[t + 3]) - de[t / 4].w);
                         p_pack[t / 2] = pack_bf16(p0, p1);
+                        p_pack[t / 2 + 1] = pack_bf16(p2, p3);
                         ds_pack[t / 2] = pack_bf16(d0, d1);
+                        ds_pack[t / 2 + 1] = pack_bf16(d2, d3);
                     }
-                    // P^T over S^T, inside this warp's own 64 columns: the 16 packed columns written here
-                    // cover fp32 columns this thread has already read
-                    tmem_st16(lane_base + COL_ST + half * 64 + cc * 16, p_pack);
+                    STAMP(15)
+                    // P^T over S^T: the 16 packed columns written here start at this thread's own first
+                    // fp32 column, which it has already read
+                    tmem_st16(lane_base + COL_ST + c0, p_pack);
                     // dS^T to shared memory: 4 chunks of 8 queries, 128-byte swizzle on the key row
+                    uint8_t* ds_row = sm.ds[i & 1][h] + ds_row_off;
 #pragma unroll
                     for (int ch = 0; ch < 4; ++ch) {
-                        const int chunk = cc * 4 + ch;
+                        const int chunk = grp * 4 + ch;
                         uint4 val = make_uint4(ds_pack[4 * ch], ds_pack[4 * ch + 1], ds_pack[4 * ch + 2], ds_pack[4 * ch + 3]);
                         *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (j & 7)) << 4)) = val;
                     }
+                    tmem_st_wait();
                 }
+                tc_fence_before();
+                fence_proxy_async_smem();
+                mbar_arrive(&sm.p_full[h]);
+                STAMP(2)
+                if (h == 0 && i > 0 && has_b) ok = drain_dq(i - 1);
             }
-            tmem_st_wait();
-            tc_fence_before();
-            fence_proxy_async_smem();
-            mbar_arrive(&sm.p_full);
-
-            // ---- drain dQ_i
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.dq_full, i & 1, abort_flag));
-            if (!ok) { if (lane == 0) report_timeout(args.status, 0x1600 + i); break; }
-            tc_fence_after();
-            {
-                const int r = j;                            // query row of the step handled by this thread
-                tmem_ld32(lane_base + COL_DQ + half * 32, s_buf);
-                tmem_ld_wait();
-                if (r < n_valid) {
-                    float* dst = args.dq_acc + ((size_t)bh * L + q0 + r) * D + half * 32;
-#pragma unroll
-                    for (int t = 0; t < 32; t += 4)
-                        red_add_v4(dst + t, __uint_as_float(s_buf[t]), __uint_as_float(s_buf[t + 1]),
-                                   __uint_as_float(s_buf[t + 2]), __uint_as_float(s_buf[t + 3]));
-                }
-            }
+            mbar_arrive(&sm.aux_empty[aslot]);      // this thread is done with the step's lse / delta
         }
+        if (ok) ok = drain_dq(n_steps - 1);
+        const int half = grp;
 
         // ---- epilogue: dK (warps 0-3) and dV (warps 4-7); the last dq_full also covers them
         if (ok) {
@@ -330,6 +463,8 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
             }
         }
+        STAMP(5)
+        if (warp == 0 && lane == 0) { STAMP_FLUSH(0, 7) STAMP_FLUSH(14, 16) }
     }
 
     tc_fence_before();
@@ -339,6 +474,18 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         tmem_dealloc(tmem, TMEM_COLS);
     }
 }
+
+#ifdef HMAR_STAMPS
+}  // namespace
+extern "C" int hmar_debug_bwd_stamps(unsigned long long* out16) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    if (cudaMemcpyFromSymbol(out16, g_bwd_stamps, sizeof(g_bwd_stamps)) != cudaSuccess) return -1;
+    unsigned long long zero[16] = {0};
+    cudaMemcpyToSymbol(g_bwd_stamps, zero, sizeof(zero));
+    return 0;
+}
+namespace {
+#endif
 
 // ------------------------------------------------------------------------------------------------
 // delta_i = sum_d dO_id * O_id  (one warp per 4 rows: 8 lanes x 16 bytes cover a row)

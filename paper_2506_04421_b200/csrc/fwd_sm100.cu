@@ -159,51 +159,62 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
     } else if (warp == 1) {
         // ================================================================== MMA issuer
-        if (lane == 0) {
-            const uint32_t q_addr = smem_u32(sm.q);
-            bool ok = mbar_wait(&sm.q_full, 0, abort_flag);
-            if (!ok) report_timeout(args.status, 0x300);
+        // The whole warp runs the control flow; one elected lane issues.  Descriptors are built once and
+        // advanced by adding (byte offset >> 4), so issuing an MMA costs a few instructions.
+        {
+            const bool leader = elect_one();
+            const uint64_t q_kd = smem_desc_sw128(smem_u32(sm.q), 16);
+            const uint64_t k_kd0 = smem_desc_sw128(smem_u32(sm.k[0]), 16);      // ring slots are 16 KB apart
+            const uint64_t v_mn0 = smem_desc_sw128(smem_u32(sm.v[0]), 1024);
+            constexpr uint32_t idesc_pv = idesc_bf16_f32(BM, D, false, true);
+            bool ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_full, 0, abort_flag));
+            if (!ok && lane == 0) report_timeout(args.status, 0x300);
             auto issue_pv = [&](int j) -> bool {      // O += P_j V_j
                 const int slot = j % NSTAGE;
                 const KvTile t = kv_tile(w, tiles0, j);
-                const int n_eff = (t.n_valid + 15) & ~15;
-                if (!mbar_wait(&sm.v_full[slot], (j / NSTAGE) & 1, abort_flag)) {
-                    report_timeout(args.status, 0x500 + j);
+                const int nk = ((t.n_valid + 15) & ~15) / 16;
+                if (!__all_sync(0xffffffffu, mbar_wait(&sm.v_full[slot], (j / NSTAGE) & 1, abort_flag))) {
+                    if (lane == 0) report_timeout(args.status, 0x500 + j);
                     return false;
                 }
                 tc_fence_after();
-                const uint32_t idesc = idesc_bf16_f32(BM, D, false, true);
-                const uint32_t v_addr = smem_u32(sm.v[slot]);
-                for (int ks = 0; ks < n_eff / 16; ++ks)
-                    mma_ts(tmem + COL_O, tmem + COL_P + ks * 8, smem_desc_sw128(v_addr + ks * 2048, 1024), idesc,
-                           (j > 0) || (ks > 0));
-                tc_commit(&sm.v_empty[slot]);
-                tc_commit(&sm.o_done);
+                if (leader) {
+                    const uint64_t vd = v_mn0 + slot * 1024;
+#pragma unroll
+                    for (int ks = 0; ks < BN / 16; ++ks)
+                        if (ks < nk)
+                            mma_ts(tmem + COL_O, tmem + COL_P + ks * 8, vd + ks * 128, idesc_pv, (j > 0) || (ks > 0));
+                    tc_commit(&sm.v_empty[slot]);
+                    tc_commit(&sm.o_done);
+                }
+                __syncwarp();
                 return true;
             };
             for (int j = 0; j < n_tiles && ok; ++j) {
                 const int slot = j % NSTAGE;
                 const KvTile t = kv_tile(w, tiles0, j);
                 const int n_eff = (t.n_valid + 15) & ~15;
-                ok = mbar_wait(&sm.k_full[slot], (j / NSTAGE) & 1, abort_flag);
-                if (!ok) { report_timeout(args.status, 0x400 + j); break; }
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.k_full[slot], (j / NSTAGE) & 1, abort_flag));
+                if (!ok) { if (lane == 0) report_timeout(args.status, 0x400 + j); break; }
                 if (j > 0) {   // S buffer free and P_{j-1} written
-                    ok = mbar_wait(&sm.p_full, (j - 1) & 1, abort_flag);
-                    if (!ok) { report_timeout(args.status, 0x600 + j); break; }
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.p_full, (j - 1) & 1, abort_flag));
+                    if (!ok) { if (lane == 0) report_timeout(args.status, 0x600 + j); break; }
                 }
                 tc_fence_after();
-                const uint32_t idesc = idesc_bf16_f32(BM, n_eff, false, false);
-                const uint32_t k_addr = smem_u32(sm.k[slot]);
-                for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(tmem + COL_S, smem_desc_sw128(q_addr + ks * 32, 16), smem_desc_sw128(k_addr + ks * 32, 16),
-                           idesc, ks > 0);
-                tc_commit(&sm.k_empty[slot]);
-                tc_commit(&sm.s_full);
+                if (leader) {
+                    const uint32_t idesc = idesc_bf16_f32(BM, n_eff, false, false);
+                    const uint64_t kd = k_kd0 + slot * 1024;
+#pragma unroll
+                    for (int ks = 0; ks < D / 16; ++ks) mma_ss(tmem + COL_S, q_kd + ks * 2, kd + ks * 2, idesc, ks > 0);
+                    tc_commit(&sm.k_empty[slot]);
+                    tc_commit(&sm.s_full);
+                }
+                __syncwarp();
                 if (j > 0) ok = issue_pv(j - 1);
             }
             if (ok) {
-                ok = mbar_wait(&sm.p_full, (n_tiles - 1) & 1, abort_flag);
-                if (!ok) report_timeout(args.status, 0x700);
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.p_full, (n_tiles - 1) & 1, abort_flag));
+                if (!ok && lane == 0) report_timeout(args.status, 0x700);
                 if (ok) {
                     tc_fence_after();
                     issue_pv(n_tiles - 1);
