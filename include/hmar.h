@@ -15,6 +15,7 @@
  *   - Entry points without suffix take bf16 tensors (raw 16-bit storage) and compute with bf16 tensor
  *     core inputs, fp32 accumulation and fp32 softmax.  The `_f32` entry points are the debug build:
  *     float tensors and plain fp32 FMA arithmetic everywhere.
+ *   - softmax_scale must be positive and finite (HMAR_ERR_BAD_ARG otherwise).
  *   - lse[b,h,i] = ln sum_j exp(softmax_scale * q_i . k_j) over the allowed j (natural log), fp32.
  *   - Every tensor pointer is DEVICE memory owned by the caller, 16-byte aligned.  `side_lens` is a
  *     HOST array read during the call.  The library allocates no per-call device memory; it owns a

@@ -53,6 +53,11 @@ __device__ int g_device_status[2];
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+static int check_scale(float softmax_scale) {
+    // the kernels take maxima before scaling, so the scale must be positive (and finite)
+    return (softmax_scale > 0.f && softmax_scale < 1e30f) ? HMAR_OK : HMAR_ERR_BAD_ARG;
+}
+
 static int check_shape(int B, int H, int D) {
     if (B <= 0 || H <= 0 || D <= 0) return HMAR_ERR_BAD_ARG;
     if ((long long)B * H > 65535) return HMAR_ERR_BAD_ARG;   // heads map to gridDim.y
@@ -109,6 +114,7 @@ static int fwd_impl(const T* q, const T* k, const T* v, T* out, float* lse, int 
     ScaleTable st;
     rc = check_sides(n_scales, side_lens, &st);
     if (rc != HMAR_OK) return rc;
+    if (check_scale(softmax_scale) != HMAR_OK) return HMAR_ERR_BAD_ARG;
     if (!q || !k || !v || !out || !lse) return HMAR_ERR_BAD_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out) || !aligned16(lse))
         return HMAR_ERR_BAD_ARG;
@@ -131,6 +137,7 @@ static int bwd_impl(const T* q, const T* k, const T* v, const T* out, const floa
     ScaleTable st;
     rc = check_sides(n_scales, side_lens, &st);
     if (rc != HMAR_OK) return rc;
+    if (check_scale(softmax_scale) != HMAR_OK) return HMAR_ERR_BAD_ARG;
     if (!q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return HMAR_ERR_BAD_ARG;
     const void* ptrs[] = {q, k, v, out, lse, dout, dq, dk, dv};
     for (const void* p : ptrs)
@@ -161,6 +168,7 @@ static int step_impl(const T* q, const T* k_prev, const T* v_prev, const T* k_cu
     int rc = check_shape(B, H, D);
     if (rc != HMAR_OK) return rc;
     if (side_cur <= 0 || side_cur > 4096 || side_prev < 0 || side_prev > 4096) return HMAR_ERR_BAD_ARG;
+    if (check_scale(softmax_scale) != HMAR_OK) return HMAR_ERR_BAD_ARG;
     if (!q || !k_cur || !v_cur || !out) return HMAR_ERR_BAD_ARG;
     if ((side_prev == 0) != (k_prev == nullptr) || (k_prev == nullptr) != (v_prev == nullptr))
         return HMAR_ERR_BAD_ARG;

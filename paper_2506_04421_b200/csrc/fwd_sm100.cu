@@ -5,13 +5,14 @@
 // IO-aware tiling with an online softmax (Sec. 4.1: the kernel extends FlashAttention), laid out for
 // Blackwell:
 //   warp 0      TMA producer: Q once, then K and V tiles of 128 keys through a shared-memory ring
-//   warp 1      issues tcgen05.mma: S = Q K^T into TMEM, then O += P V with P read from TMEM
-//   warps 2-5   one query row per thread: read S from TMEM, mask, running max / sum in fp32,
-//               write P (bf16) back to TMEM, rescale O only when the running max grew by > 2^8,
-//               and finally normalise O and write out / lse
-// TMEM columns: S fp32 [0,128), P bf16 [128,192), O fp32 [192,256).  Two blocks fit on one SM
-// (256 TMEM columns and ~82 KB of shared memory each), so one block's softmax overlaps the other
-// block's matrix products.
+//   warp 1      issues tcgen05.mma.  Q is copied to TMEM once and is the A operand of S = Q K^T; a key
+//               tile is handled as two halves of 64 keys with their own S columns and barriers, so the
+//               tensor core computes one half while the softmax warps work on the other.  P replaces S
+//               in place (bf16) and is the TMEM A operand of O += P V.
+//   warps 2-5   one query row per thread.  A half's 64 logits are read from TMEM once; the running
+//               maximum is kept unless the half exceeds it by more than 2^8 (then O and the row sum are
+//               rescaled first), P = 2^(s - m) goes back to TMEM as bf16.
+// TMEM columns: S/P half a [0,64), half b [64,128), O [128,192), Q [192,224).  Two blocks fit on one SM.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -28,21 +29,22 @@ using namespace ptx;
 
 constexpr int BM = 128;              // query rows per block
 constexpr int BN = 128;              // keys per tile
+constexpr int HN = 64;               // keys per half tile
 constexpr int D = kHeadDim;
 constexpr int NSTAGE = 2;
 constexpr int TILE_BYTES = BN * D * 2;          // 16 KB
 constexpr int NUM_THREADS = 192;
 constexpr uint32_t TMEM_COLS = 256;
-constexpr uint32_t COL_S = 0, COL_P = 128, COL_O = 192;
+constexpr uint32_t COL_S = 0, COL_O = 128, COL_Q = 192;
 constexpr float kRescaleThreshold = 8.0f;       // in log2 units
 
 struct __align__(1024) SharedStorage {
     uint8_t q[TILE_BYTES];
     uint8_t k[NSTAGE][TILE_BYTES];
     uint8_t v[NSTAGE][TILE_BYTES];
-    uint64_t q_full;
+    uint64_t q_full, q_tmem;
     uint64_t k_full[NSTAGE], k_empty[NSTAGE], v_full[NSTAGE], v_empty[NSTAGE];
-    uint64_t s_full, p_full, o_done;
+    uint64_t s_full[2], p_full[2], pv_done;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -65,6 +67,12 @@ __device__ __forceinline__ KvTile kv_tile(const FwdWork& w, int tiles0, int j) {
         t.n_valid = min(BN, w.s1_end - t.coord);
     }
     return t;
+}
+
+// columns issued for half h of a tile with n_valid keys (multiple of 16, 0 if the half is empty)
+__device__ __forceinline__ int half_cols(int n_valid, int h) {
+    const int n_eff = (n_valid + 15) & ~15;
+    return h == 0 ? min(n_eff, HN) : max(n_eff - HN, 0);
 }
 
 __device__ __forceinline__ void report_timeout(int* status, int where) {
@@ -108,15 +116,18 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     if (threadIdx.x == 0) {
         sm.abort_flag = 0;
         mbar_init(&sm.q_full, 1);
+        mbar_init(&sm.q_tmem, 128);
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(&sm.k_full[s], 1);
             mbar_init(&sm.k_empty[s], 1);
             mbar_init(&sm.v_full[s], 1);
             mbar_init(&sm.v_empty[s], 1);
         }
-        mbar_init(&sm.s_full, 1);
-        mbar_init(&sm.p_full, 128);
-        mbar_init(&sm.o_done, 1);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(&sm.s_full[h], 1);
+            mbar_init(&sm.p_full[h], 128);
+        }
+        mbar_init(&sm.pv_done, 1);
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -161,65 +172,76 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         // ================================================================== MMA issuer
         // The whole warp runs the control flow; one elected lane issues.  Descriptors are built once and
         // advanced by adding (byte offset >> 4), so issuing an MMA costs a few instructions.
-        {
-            const bool leader = elect_one();
-            const uint64_t q_kd = smem_desc_sw128(smem_u32(sm.q), 16);
-            const uint64_t k_kd0 = smem_desc_sw128(smem_u32(sm.k[0]), 16);      // ring slots are 16 KB apart
-            const uint64_t v_mn0 = smem_desc_sw128(smem_u32(sm.v[0]), 1024);
-            constexpr uint32_t idesc_pv = idesc_bf16_f32(BM, D, false, true);
-            bool ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_full, 0, abort_flag));
-            if (!ok && lane == 0) report_timeout(args.status, 0x300);
-            auto issue_pv = [&](int j) -> bool {      // O += P_j V_j
-                const int slot = j % NSTAGE;
-                const KvTile t = kv_tile(w, tiles0, j);
-                const int nk = ((t.n_valid + 15) & ~15) / 16;
-                if (!__all_sync(0xffffffffu, mbar_wait(&sm.v_full[slot], (j / NSTAGE) & 1, abort_flag))) {
-                    if (lane == 0) report_timeout(args.status, 0x500 + j);
-                    return false;
-                }
-                tc_fence_after();
-                if (leader) {
-                    const uint64_t vd = v_mn0 + slot * 1024;
+        const bool leader = elect_one();
+        const uint64_t k_kd0 = smem_desc_sw128(smem_u32(sm.k[0]), 16);      // ring slots are 16 KB apart
+        const uint64_t v_mn0 = smem_desc_sw128(smem_u32(sm.v[0]), 1024);
+        constexpr uint32_t idesc_pv = idesc_bf16_f32(BM, D, false, true);
+        int p_seen[2] = {0, 0};                                 // completed phases of p_full[h] consumed so far
+        bool ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_tmem, 0, abort_flag));
+        if (!ok && lane == 0) report_timeout(args.status, 0x300);
+
+        // S_h = Q K_h^T for half h of tile j (Q from TMEM, 64 keys of the tile from shared memory)
+        auto issue_s = [&](int j, int h) -> bool {
+            const int slot = j % NSTAGE;
+            const int n = half_cols(kv_tile(w, tiles0, j).n_valid, h);
+            if (n == 0) return true;
+            if (h == 0 && !__all_sync(0xffffffffu, mbar_wait(&sm.k_full[slot], (j / NSTAGE) & 1, abort_flag))) {
+                if (lane == 0) report_timeout(args.status, 0x400 + j);
+                return false;
+            }
+            tc_fence_after();
+            if (leader) {
+                const uint32_t idesc = idesc_bf16_f32(BM, n, false, false);
+                const uint64_t kd = k_kd0 + slot * 1024 + h * 512;              // + 64 rows
 #pragma unroll
-                    for (int ks = 0; ks < BN / 16; ++ks)
-                        if (ks < nk)
-                            mma_ts(tmem + COL_O, tmem + COL_P + ks * 8, vd + ks * 128, idesc_pv, (j > 0) || (ks > 0));
-                    tc_commit(&sm.v_empty[slot]);
-                    tc_commit(&sm.o_done);
-                }
-                __syncwarp();
-                return true;
-            };
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int slot = j % NSTAGE;
-                const KvTile t = kv_tile(w, tiles0, j);
-                const int n_eff = (t.n_valid + 15) & ~15;
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm.k_full[slot], (j / NSTAGE) & 1, abort_flag));
-                if (!ok) { if (lane == 0) report_timeout(args.status, 0x400 + j); break; }
-                if (j > 0) {   // S buffer free and P_{j-1} written
-                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.p_full, (j - 1) & 1, abort_flag));
-                    if (!ok) { if (lane == 0) report_timeout(args.status, 0x600 + j); break; }
-                }
-                tc_fence_after();
-                if (leader) {
-                    const uint32_t idesc = idesc_bf16_f32(BM, n_eff, false, false);
-                    const uint64_t kd = k_kd0 + slot * 1024;
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ts(tmem + COL_S + h * HN, tmem + COL_Q + ks * 8, kd + ks * 2, idesc, ks > 0);
+                tc_commit(&sm.s_full[h]);
+            }
+            __syncwarp();
+            return true;
+        };
+        // O += P_h V_h for half h of tile j; the tile's last half releases its K and V slots
+        auto issue_pv = [&](int j, int h) -> bool {
+            const int slot = j % NSTAGE;
+            const int n_valid = kv_tile(w, tiles0, j).n_valid;
+            const int n = half_cols(n_valid, h);
+            if (n == 0) return true;
+            const int par = h == 0 ? (p_seen[0]++ & 1) : (p_seen[1]++ & 1);
+            if (!__all_sync(0xffffffffu, mbar_wait(&sm.p_full[h], par, abort_flag))) {
+                if (lane == 0) report_timeout(args.status, 0x600 + j);
+                return false;
+            }
+            if (h == 0 && !__all_sync(0xffffffffu, mbar_wait(&sm.v_full[slot], (j / NSTAGE) & 1, abort_flag))) {
+                if (lane == 0) report_timeout(args.status, 0x500 + j);
+                return false;
+            }
+            tc_fence_after();
+            if (leader) {
+                const int nk = n / 16;
+                const uint64_t vd = v_mn0 + slot * 1024 + h * 512;
+                const bool first = (j == 0) && (h == 0);
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) mma_ss(tmem + COL_S, q_kd + ks * 2, kd + ks * 2, idesc, ks > 0);
+                for (int ks = 0; ks < HN / 16; ++ks)
+                    if (ks < nk)
+                        mma_ts(tmem + COL_O, tmem + COL_S + h * HN + ks * 8, vd + ks * 128, idesc_pv, !first || (ks > 0));
+                tc_commit(&sm.pv_done);
+                if (h == 1 || half_cols(n_valid, 1) == 0) {      // last half of the tile
                     tc_commit(&sm.k_empty[slot]);
-                    tc_commit(&sm.s_full);
-                }
-                __syncwarp();
-                if (j > 0) ok = issue_pv(j - 1);
-            }
-            if (ok) {
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm.p_full, (n_tiles - 1) & 1, abort_flag));
-                if (!ok && lane == 0) report_timeout(args.status, 0x700);
-                if (ok) {
-                    tc_fence_after();
-                    issue_pv(n_tiles - 1);
+                    tc_commit(&sm.v_empty[slot]);
                 }
             }
+            __syncwarp();
+            return true;
+        };
+
+        if (ok) ok = issue_s(0, 0);
+        if (ok) ok = issue_s(0, 1);
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            ok = issue_pv(j, 0);
+            if (ok && j + 1 < n_tiles) ok = issue_s(j + 1, 0);
+            if (ok) ok = issue_pv(j, 1);
+            if (ok && j + 1 < n_tiles) ok = issue_s(j + 1, 1);
         }
     } else {
         // ================================================================== softmax + epilogue
@@ -237,91 +259,124 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const float sl2 = args.scale_log2;
         float m_used = -INFINITY, l = 0.f;
         bool ok = true;
-        uint32_t buf[32];
+        int pv_issued = 0;                                     // halves handed to the tensor core so far
+        int s_seen[2] = {0, 0};                                // completed phases of s_full[h] consumed so far
+        uint32_t b0[32], b1[32];
 
-        for (int j = 0; j < n_tiles; ++j) {
+        // ---- Q row to TMEM (A operand of S = Q K^T): undo the 128-byte swizzle of the TMA tile
+        ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_full, 0, abort_flag));
+        if (!ok && lane == 0) report_timeout(args.status, 0x700);
+        if (ok) {
+            const uint8_t* qrow = sm.q + r * 128;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint4 val = *reinterpret_cast<const uint4*>(qrow + ((c ^ (r & 7)) << 4));
+                b0[4 * c] = val.x; b0[4 * c + 1] = val.y; b0[4 * c + 2] = val.z; b0[4 * c + 3] = val.w;
+            }
+            tmem_st32(lane_base + COL_Q, b0);
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(&sm.q_tmem);
+        }
+
+        for (int j = 0; j < n_tiles && ok; ++j) {
             const KvTile t = kv_tile(w, tiles0, j);
-            const int n_eff = (t.n_valid + 15) & ~15;
-            const int n_chunks = (n_eff + 31) / 32;
-            const bool need_mask = (!w.uniform) || (t.n_valid < n_chunks * 32);
-            // key c of the tile is visible iff c in [c_lo, c_hi)
+            // key c of the tile is visible to this row iff c in [c_lo, c_hi)
             const int c_lo = w.uniform ? 0 : max(lo - t.coord, 0);
             const int c_hi = w.uniform ? t.n_valid : min(hi - t.coord, t.n_valid);
 
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full, j & 1, abort_flag));
-            if (!ok) { if (lane == 0) report_timeout(args.status, 0x800 + j); break; }
-            tc_fence_after();
+            for (int h = 0; h < 2 && ok; ++h) {
+                const int n = half_cols(t.n_valid, h);
+                if (n == 0) break;
+                const int col0 = h * HN;                           // first key of the half inside the tile
+                const bool two = n > 32;                           // second 32-column chunk present
+                const bool need_mask = (!w.uniform) || (t.n_valid < col0 + (two ? 64 : 32));
+                const uint32_t s_addr = lane_base + COL_S + col0;
 
-            // ---- pass 1: row maximum of the scaled logits (log2 units)
-            float mx = -INFINITY;
-            for (int ch = 0; ch < n_chunks; ++ch) {
-                tmem_ld32(lane_base + COL_S + ch * 32, buf);
+                const int par = h == 0 ? (s_seen[0]++ & 1) : (s_seen[1]++ & 1);
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[h], par, abort_flag));
+                if (!ok) { if (lane == 0) report_timeout(args.status, 0x800 + j); break; }
+                tc_fence_after();
+
+                tmem_ld32(s_addr, b0);
+                if (two) tmem_ld32(s_addr + 32, b1);
                 tmem_ld_wait();
+
+                // masked logits become -inf once, so the maximum and the exponentials treat them alike
                 if (need_mask) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
-                        const int c = ch * 32 + i;
-                        const float s = __uint_as_float(buf[i]) * sl2;
-                        mx = fmaxf(mx, (c >= c_lo && c < c_hi) ? s : -INFINITY);
+                        if (!(col0 + i >= c_lo && col0 + i < c_hi)) b0[i] = 0xff800000u;
+                        if (!(col0 + 32 + i >= c_lo && col0 + 32 + i < c_hi)) b1[i] = 0xff800000u;
                     }
-                } else {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(buf[i]) * sl2);
                 }
-            }
-            const float m_new = fmaxf(m_used, mx);
-            const float m_old = m_used;
-            const bool want = (j == 0) || (m_new > m_used + kRescaleThreshold);
-            const bool any = __any_sync(0xffffffffu, want);
+                float mx = -INFINITY;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(b0[i]));
+                if (two) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(b1[i]));
+                }
+                mx *= sl2;                                          // softmax_scale > 0
 
-            if (j > 0) {    // P buffer free again, O not being accumulated into
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_done, (j - 1) & 1, abort_flag));
-                if (!ok) { if (lane == 0) report_timeout(args.status, 0x900 + j); break; }
-                tc_fence_after();
-            }
-            if (any) {
-                m_used = m_new;
-                if (j > 0) {
-                    const float f = (m_old == -INFINITY) ? 0.f : ex2(m_old - m_used);
+                // Keep the running maximum unless this half exceeds it by more than the threshold.
+                const bool grow = mx > m_used + kRescaleThreshold;  // false for -inf > -inf
+                if (__any_sync(0xffffffffu, grow)) {
+                    // O must be quiet: wait for every P V product handed over so far
+                    if (pv_issued > 0) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(&sm.pv_done, (pv_issued - 1) & 1, abort_flag));
+                        if (!ok) { if (lane == 0) report_timeout(args.status, 0x900 + j); break; }
+                        tc_fence_after();
+                    }
+                    const float m_new = fmaxf(m_used, mx);
+                    const float f = (m_used == -INFINITY) ? 0.f : ex2(m_used - m_new);
+                    m_used = m_new;
                     l *= f;
+                    if (pv_issued > 0) {
+                        uint32_t o[32];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        tmem_ld32(lane_base + COL_O + h * 32, buf);
-                        tmem_ld_wait();
+                        for (int hh = 0; hh < 2; ++hh) {
+                            tmem_ld32(lane_base + COL_O + hh * 32, o);
+                            tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) buf[i] = __float_as_uint(__uint_as_float(buf[i]) * f);
-                        tmem_st32(lane_base + COL_O + h * 32, buf);
+                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                            tmem_st32(lane_base + COL_O + hh * 32, o);
+                        }
                     }
                 }
-            }
-            const float m_sub = (m_used == -INFINITY) ? 0.f : m_used;
+                const float m_sub = (m_used == -INFINITY) ? 0.f : m_used;
 
-            // ---- pass 2: P = 2^(s - m), row sum, bf16 P back to TMEM
-            for (int ch = 0; ch < n_chunks; ++ch) {
-                tmem_ld32(lane_base + COL_S + ch * 32, buf);
-                tmem_ld_wait();
+                // P = 2^(s * scale - m): fp32 row sum, bf16 P written over the S columns already read
                 uint32_t packed[16];
+                float l_add = 0.f;
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    float p0 = ex2(fmaf(__uint_as_float(buf[i]), sl2, -m_sub));
-                    float p1 = ex2(fmaf(__uint_as_float(buf[i + 1]), sl2, -m_sub));
-                    if (need_mask) {
-                        const int c = ch * 32 + i;
-                        p0 = (c >= c_lo && c < c_hi) ? p0 : 0.f;
-                        p1 = (c + 1 >= c_lo && c + 1 < c_hi) ? p1 : 0.f;
-                    }
-                    l += p0 + p1;
+                    const float p0 = ex2(fmaf(__uint_as_float(b0[i]), sl2, -m_sub));
+                    const float p1 = ex2(fmaf(__uint_as_float(b0[i + 1]), sl2, -m_sub));
+                    l_add += p0 + p1;
                     packed[i / 2] = pack_bf16(p0, p1);
                 }
-                tmem_st16(lane_base + COL_P + ch * 16, packed);
+                tmem_st16(s_addr, packed);
+                if (two) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 2) {
+                        const float p0 = ex2(fmaf(__uint_as_float(b1[i]), sl2, -m_sub));
+                        const float p1 = ex2(fmaf(__uint_as_float(b1[i + 1]), sl2, -m_sub));
+                        l_add += p0 + p1;
+                        packed[i / 2] = pack_bf16(p0, p1);
+                    }
+                    tmem_st16(s_addr + 16, packed);
+                }
+                l += l_add;
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(&sm.p_full[h]);
+                ++pv_issued;
             }
-            tmem_st_wait();
-            tc_fence_before();
-            mbar_arrive(&sm.p_full);
         }
 
         if (ok) {
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_done, (n_tiles - 1) & 1, abort_flag));
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.pv_done, (pv_issued - 1) & 1, abort_flag));
             if (!ok && lane == 0) report_timeout(args.status, 0xA00);
         }
         if (ok) {
@@ -330,18 +385,18 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             __nv_bfloat16* orow = args.out + ((size_t)bh * args.n_q_rows + row) * D;
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                tmem_ld32(lane_base + COL_O + h * 32, buf);
+                tmem_ld32(lane_base + COL_O + h * 32, b0);
                 tmem_ld_wait();
                 if (row_ok) {
                     uint4* dst = reinterpret_cast<uint4*>(orow + h * 32);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(buf[8 * i + 0]) * inv, __uint_as_float(buf[8 * i + 1]) * inv);
-                        o.y = pack_bf16(__uint_as_float(buf[8 * i + 2]) * inv, __uint_as_float(buf[8 * i + 3]) * inv);
-                        o.z = pack_bf16(__uint_as_float(buf[8 * i + 4]) * inv, __uint_as_float(buf[8 * i + 5]) * inv);
-                        o.w = pack_bf16(__uint_as_float(buf[8 * i + 6]) * inv, __uint_as_float(buf[8 * i + 7]) * inv);
-                        dst[i] = o;
+                        uint4 v4;
+                        v4.x = pack_bf16(__uint_as_float(b0[8 * i + 0]) * inv, __uint_as_float(b0[8 * i + 1]) * inv);
+                        v4.y = pack_bf16(__uint_as_float(b0[8 * i + 2]) * inv, __uint_as_float(b0[8 * i + 3]) * inv);
+                        v4.z = pack_bf16(__uint_as_float(b0[8 * i + 4]) * inv, __uint_as_float(b0[8 * i + 5]) * inv);
+                        v4.w = pack_bf16(__uint_as_float(b0[8 * i + 6]) * inv, __uint_as_float(b0[8 * i + 7]) * inv);
+                        dst[i] = v4;
                     }
                 }
             }

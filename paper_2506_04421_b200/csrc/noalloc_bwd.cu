@@ -63,6 +63,7 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
                                      float softmax_scale, void* stream) {
     if (B <= 0 || H <= 0 || D <= 0 || (long long)B * H > 65535) return HMAR_ERR_BAD_ARG;
     if (D != kHeadDim) return HMAR_ERR_UNSUPPORTED;
+    if (!(softmax_scale > 0.f && softmax_scale < 1e30f)) return HMAR_ERR_BAD_ARG;
     if (n_scales <= 0 || n_scales > HMAR_MAX_SCALES || side_lens == nullptr) return HMAR_ERR_BAD_ARG;
     long long L = 0;
     for (int s = 0; s < n_scales; ++s) {

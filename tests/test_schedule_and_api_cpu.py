@@ -66,11 +66,12 @@ def test_library_exports_every_declared_symbol():
         assert getattr(L, name) is not None
 
 
-def _call_fwd(q=1 << 12, k=1 << 12, v=1 << 12, out=1 << 12, lse=1 << 12, B=1, H=1, D=64, sides=(1, 2)):
+def _call_fwd(q=1 << 12, k=1 << 12, v=1 << 12, out=1 << 12, lse=1 << 12, B=1, H=1, D=64, sides=(1, 2),
+              scale=0.125):
     arr = (ctypes.c_int * max(len(sides), 1))(*sides)
     vp = ctypes.c_void_p
     return hmar.lib().hmar_attn_fwd(vp(q), vp(k), vp(v), vp(out), vp(lse), B, H, D, len(sides), arr,
-                                    0.125, None)
+                                    scale, None)
 
 
 def test_argument_errors_are_reported_before_any_launch():
@@ -84,6 +85,10 @@ def test_argument_errors_are_reported_before_any_launch():
     assert _call_fwd(sides=(1, -3)) == hmar.HMAR_ERR_BAD_ARG
     assert _call_fwd(sides=tuple([1] * 65)) == hmar.HMAR_ERR_BAD_ARG
     assert _call_fwd(B=70000) == hmar.HMAR_ERR_BAD_ARG
+    assert _call_fwd(scale=0.0) == hmar.HMAR_ERR_BAD_ARG
+    assert _call_fwd(scale=-0.125) == hmar.HMAR_ERR_BAD_ARG
+    assert _call_fwd(scale=float("inf")) == hmar.HMAR_ERR_BAD_ARG
+    assert _call_fwd(scale=float("nan")) == hmar.HMAR_ERR_BAD_ARG
     assert hmar.hmar_attn_bwd_workspace_bytes(1, 1, 32, (1, 2)) == 0
     assert hmar.hmar_attn_bwd_workspace_bytes(2, 3, 64, (1, 2)) >= 2 * 3 * 5 * (64 + 1) * 4
     with pytest.raises(hmar.HmarError):
