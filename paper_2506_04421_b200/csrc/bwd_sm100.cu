@@ -5,22 +5,29 @@
 //   P = exp(scale * Q K^T - lse),  dV = P^T dO,  dP = dO V^T,  dS = P o (dP - delta),
 //   dQ = scale * dS K,  dK = scale * dS^T Q,  delta_i = sum_d dO_id O_id.
 //
-// Main kernel: one block owns one tile of up to 128 key rows of one head and walks over the
-// contiguous range of query rows that may see them under the mask (queries of the keys' own scale and
-// of the next scale; paper Sec. 4.1, Fig. attn-mask), 128 queries at a time:
-//   warp 8      TMA producer: K, V once; then Q_i, dO_i through a 3-stage ring
-//   warp 10     loads lse_i, delta_i with plain loads (their row offsets are not 16-byte aligned) into
+// Main kernel: persistent blocks, one per SM.  A work item is one tile of up to 128 key rows of one
+// head; the block walks over the contiguous range of query rows that may see them under the mask
+// (queries of the keys' own scale and of the next scale; paper Sec. 4.1, Fig. attn-mask), 128 queries
+// (one step) at a time.  A step is split into two halves of 64 queries with their own TMEM columns and
+// barriers; each half belongs to one compute warpgroup, so the two warpgroups and the tensor core work
+// on different halves at the same time.
+//   warps 0-3   compute warpgroup of half 0: one key row per thread, 64 query columns.  P^T and dS^T
+//               in fp32; P^T (bf16) goes back to TMEM over S^T, dS^T (bf16) goes to TMEM over dP^T
+//               (A operand of dK) and to shared memory (A operand of dQ)
+//   warps 4-7   the same for half 1
+//   warps 8-11  drain dQ_i from TMEM through a staging buffer into the fp32 accumulator with bulk tensor
+//               reductions (cp.reduce.async.bulk.tensor)
+//   warp 12     TMA producer: K, V per item; Q_i, dO_i through a 3-stage ring that runs across items
+//   warp 13     issues tcgen05.mma.  K and V are copied to TMEM once per item and are the A operands of
+//               S^T = K Q_i^T and dP^T = V dO_i^T; dV += P^T dO_i and dK += dS^T Q_i read their A operand
+//               from TMEM too; dQ_i = dS K reads dS from shared memory as an MN-major operand
+//   warp 14     loads lse_i, delta_i with plain loads (their row offsets are not 16-byte aligned) into
 //               an 8-deep ring
-//   warp 9      issues tcgen05.mma: S^T = K Q_i^T and dP^T = V dO_i^T into TMEM; after the compute
-//               warps are done: dV += P^T dO_i (P^T read from TMEM), dK += dS^T Q_i and
-//               dQ_i = dS K (dS read from shared memory, once as a K-major and once as an
-//               MN-major operand)
-//   warps 0-7   one key row per thread, two threads per row splitting the 128 query columns:
-//               P^T and dS^T in fp32, P^T (bf16) back to TMEM over S^T, dS^T (bf16) to shared memory;
-//               then they drain dQ_i from TMEM into the fp32 accumulator with vector atomics
-// TMEM columns: S^T [0,128) (P^T of queries 0-63 over columns [0,32), of queries 64-127 over
-// [64,96)), dP^T [128,256), dK [256,320), dV [320,384), dQ_i [384,448).
-// dK and dV stay in TMEM for the whole block and are written once at the end.
+// TMEM columns: S^T [0,128) (half h at h*64; P^T of half h over its first 32 columns), dP^T [128,256)
+// (dS^T likewise), dK [256,320), dV [320,384), dQ_i [384,448), K [448,480), V [480,512).
+// dK and dV stay in TMEM for a whole item and are written once at its end.
+// Registers: the block starts with 128 per thread; the compute warpgroups raise theirs and the other
+// two warpgroups lower theirs (setmaxnreg) within the same total.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -35,17 +42,26 @@ namespace {
 
 using namespace ptx;
 
-constexpr int BKV = 128;             // key rows per block
+constexpr int BKV = 128;             // key rows per item
 constexpr int BQ = 128;              // query rows per step
+constexpr int HQ = 64;               // query rows per half step
 constexpr int D = kHeadDim;
 constexpr int NSTAGE = 3;
 constexpr int AUX_STAGES = 8;        // ring of lse / delta rows, loaded this many steps ahead
 constexpr int TILE_BYTES = 128 * D * 2;          // 16 KB
-constexpr int NUM_COMPUTE_WARPS = 8;
-constexpr int PRODUCER_WARP = 8, MMA_WARP = 9, AUX_WARP = 10;
-constexpr int NUM_THREADS = 352;
+constexpr int WORK_CACHE = 64;       // work tiles of a head kept in shared memory
+constexpr int NUM_COMPUTE_THREADS = 256;
+constexpr int DRAIN_WARP0 = 8, PRODUCER_WARP = 12, MMA_WARP = 13, AUX_WARP = 14;
+constexpr int NUM_THREADS = 512;
+#ifndef X_RC
+#define X_RC 176
+#define X_RD 64
+#define X_RM 96
+#endif
+constexpr int REGS_COMPUTE = X_RC, REGS_DRAIN = X_RD, REGS_MISC = X_RM;
+static_assert(2 * REGS_COMPUTE + REGS_DRAIN + REGS_MISC == 4 * 128, "register budget of the block");
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t COL_ST = 0, COL_DPT = 128, COL_DK = 256, COL_DV = 320, COL_DQ = 384;
+constexpr uint32_t COL_ST = 0, COL_DPT = 128, COL_DK = 256, COL_DV = 320, COL_DQ = 384, COL_K = 448, COL_V = 480;
 
 struct __align__(1024) SharedStorage {
     uint8_t k[TILE_BYTES];
@@ -53,13 +69,17 @@ struct __align__(1024) SharedStorage {
     uint8_t q[NSTAGE][TILE_BYTES];
     uint8_t dout[NSTAGE][TILE_BYTES];
     uint8_t ds[2][2][TILE_BYTES];           // dS^T, double buffered: [step parity][64-query half][key row][64 queries], 128B swizzle
+    uint8_t dq_stage[TILE_BYTES];           // 128 query rows x 32 fp32 columns of dQ_i on their way to the accumulator, 128B swizzle
     float lse2[AUX_STAGES][BQ];             // lse * log2(e); +inf for query rows outside the range
     float delta[AUX_STAGES][BQ];
-    uint64_t kv_full;
+    uint64_t kv_full, kv_tmem;
     uint64_t qdo_full[NSTAGE], q_empty[NSTAGE], aux_full[AUX_STAGES], aux_empty[AUX_STAGES];
-    uint64_t s_full[2], p_full[2], dq_full;   // [half of the step]
+    uint64_t s_full[2], p_full[2];            // [half of the step]
+    uint64_t dq_full, dq_empty, acc_full, acc_empty, drain_sync;
+    BwdWork work[WORK_CACHE];               // the head's work list (its first WORK_CACHE tiles)
     uint32_t tmem_base;
     int abort_flag;
+    int item_begin, item_end;
 };
 
 __device__ __forceinline__ void report_timeout(int* status, int where) {
@@ -69,32 +89,55 @@ __device__ __forceinline__ void report_timeout(int* status, int where) {
     }
 }
 
-__device__ __forceinline__ void red_add_v4(float* addr, float a, float b, float c, float d) {
-    asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(a), "f"(b), "f"(c),
-                 "f"(d)
-                 : "memory");
-}
-
-#ifdef HMAR_STAMPS
-// Developer build only: per-phase clock totals of compute warp 0 and of the MMA thread, summed over blocks.
-__device__ unsigned long long g_bwd_stamps[16];
-#define STAMP_DECL unsigned long long st_acc[16] = {0}; long long st_t = clock64();
-#define STAMP(idx) { long long st_n = clock64(); st_acc[idx] += (unsigned long long)(st_n - st_t); st_t = st_n; }
-#define STAMP_FLUSH(lo, hi) { for (int st_i = lo; st_i < hi; ++st_i) atomicAdd(&g_bwd_stamps[st_i], st_acc[st_i]); }
-#else
-#define STAMP_DECL
-#define STAMP(idx) {}
-#define STAMP_FLUSH(lo, hi) {}
-#endif
-
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
+
+// Adds a [128 rows x 32 fp32] tile in shared memory (128-byte swizzle) to global memory at (column c0, row c1).
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* m, const void* smem_src, int c0, int c1) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+template <int N> __device__ __forceinline__ void reg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N> __device__ __forceinline__ void reg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
+// One row of a 128-byte-swizzled [128 rows x 64 bf16] tile, as 32 packed words in row order.
+__device__ __forceinline__ void load_swizzled_row(const uint8_t* tile, int r, uint32_t (&dst)[32]) {
+    const uint8_t* row = tile + r * 128;
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const uint4 val = *reinterpret_cast<const uint4*>(row + ((c ^ (r & 7)) << 4));
+        dst[4 * c] = val.x; dst[4 * c + 1] = val.y; dst[4 * c + 2] = val.z; dst[4 * c + 3] = val.w;
+    }
+}
+
+// Work items of one block.  Item g is tile g % n_work of head g / n_work; items are ordered head by
+// head (a head's Q and dO tiles stay in L2 while its key tiles are processed) and every block takes a
+// contiguous run of items of about the same total cost (steps plus a constant per item).
+__device__ __forceinline__ int first_item_at_cost(const BwdArgs& args, long long cost) {
+    const long long head = cost / args.head_cost;
+    const int rem = (int)(cost - head * args.head_cost);
+    int lo = 0, hi = args.n_work;                       // first tile whose starting cost is >= rem
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(&args.work[mid].cost_begin) >= rem) hi = mid; else lo = mid + 1;
+    }
+    return (int)head * args.n_work + lo;
 }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
-                   const BwdArgs args) {
+                   const __grid_constant__ CUtensorMap map_dq, const BwdArgs args) {
     extern __shared__ uint8_t smem_raw[];
     SharedStorage& sm = *reinterpret_cast<SharedStorage*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -103,29 +146,37 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
     if (args.status != nullptr && *reinterpret_cast<volatile int*>(args.status) != 0) return;
 
-    const int bh = blockIdx.x / args.n_work;
-    const BwdWork w = args.work[blockIdx.x % args.n_work];
-    const int n_steps = (w.q_end - w.q_begin + BQ - 1) / BQ;
     const int L = args.L;
+    const int n_work = args.n_work;
 
     if (threadIdx.x == 0) {
         sm.abort_flag = 0;
         mbar_init(&sm.kv_full, 1);
+        mbar_init(&sm.kv_tmem, NUM_COMPUTE_THREADS);
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(&sm.qdo_full[s], 1);
             mbar_init(&sm.q_empty[s], 1);
         }
         for (int s = 0; s < AUX_STAGES; ++s) {
             mbar_init(&sm.aux_full[s], 32);
-            mbar_init(&sm.aux_empty[s], NUM_COMPUTE_WARPS * 32);
+            mbar_init(&sm.aux_empty[s], NUM_COMPUTE_THREADS);
         }
         for (int h = 0; h < 2; ++h) {
             mbar_init(&sm.s_full[h], 1);
-            mbar_init(&sm.p_full[h], NUM_COMPUTE_WARPS * 32);
+            mbar_init(&sm.p_full[h], NUM_COMPUTE_THREADS / 2);
         }
         mbar_init(&sm.dq_full, 1);
+        mbar_init(&sm.dq_empty, 128);
+        mbar_init(&sm.acc_full, 1);
+        mbar_init(&sm.acc_empty, NUM_COMPUTE_THREADS);
+        mbar_init(&sm.drain_sync, 128);
         fence_mbar_init();
+        const long long total = (long long)args.n_heads * args.head_cost;
+        sm.item_begin = first_item_at_cost(args, total * blockIdx.x / gridDim.x);
+        sm.item_end = blockIdx.x + 1 == gridDim.x ? args.n_heads * n_work
+                                                  : first_item_at_cost(args, total * (blockIdx.x + 1) / gridDim.x);
     }
+    for (int t = threadIdx.x; t < min(n_work, WORK_CACHE); t += NUM_THREADS) sm.work[t] = args.work[t];
     if (warp == MMA_WARP) {
         tmem_alloc(&sm.tmem_base, TMEM_COLS);
         tmem_relinquish();
@@ -134,337 +185,432 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
+    const int item_begin = sm.item_begin, item_end = sm.item_end;
     volatile int* abort_flag = &sm.abort_flag;
 
-    if (warp == PRODUCER_WARP) {
-        // ================================================================== producer
-        if (lane == 0) {
-            prefetch_tensormap(&map_q);
-            prefetch_tensormap(&map_k);
-            prefetch_tensormap(&map_v);
-            prefetch_tensormap(&map_do);
-            mbar_arrive_expect_tx(&sm.kv_full, 2 * TILE_BYTES);
-            tma_load_3d(sm.k, &map_k, &sm.kv_full, 0, w.row_begin, bh);
-            tma_load_3d(sm.v, &map_v, &sm.kv_full, 0, w.row_begin, bh);
-        }
-        bool ok = true;
-        if (lane == 0) {
-            for (int i = 0; i < n_steps; ++i) {
-                const int slot = i % NSTAGE;
-                const int q0 = w.q_begin + i * BQ;
-                if (i >= NSTAGE) {
-                    ok = mbar_wait(&sm.q_empty[slot], ((i / NSTAGE) & 1) ^ 1, abort_flag);
-                    if (!ok) { report_timeout(args.status, 0x1100 + i); break; }
-                }
-                mbar_arrive_expect_tx(&sm.qdo_full[slot], 2 * TILE_BYTES);
-                tma_load_3d(sm.q[slot], &map_q, &sm.qdo_full[slot], 0, q0, bh);
-                tma_load_3d(sm.dout[slot], &map_do, &sm.qdo_full[slot], 0, q0, bh);
-            }
-        }
-        if (!ok && lane == 0) {
-            const uint64_t t0 = globaltimer_ns();
-            while (globaltimer_ns() - t0 < 2000000ull) { }
-        }
-    } else if (warp == AUX_WARP) {
-        // ================================================================== lse / delta loader
-        // lse and delta rows of step i go to ring slot i % AUX_STAGES, several steps ahead of their use
-        // (plain loads: their row offsets are not 16-byte aligned, so TMA cannot fetch them).
-        STAMP_DECL
-        for (int i = 0; i < n_steps; ++i) {
-            const int aslot = i % AUX_STAGES;
-            STAMP(13)
-            if (i >= AUX_STAGES) {
-                const bool ok = __all_sync(0xffffffffu,
-                                           mbar_wait(&sm.aux_empty[aslot], ((i / AUX_STAGES) & 1) ^ 1, abort_flag));
-                if (!ok) { if (lane == 0) report_timeout(args.status, 0x1700 + i); break; }
-            }
-            STAMP(12)
-            const int q0 = w.q_begin + i * BQ;
-            // all loads first, then the stores: stores to shared memory in between would serialise them
-            float lv[BQ / 32], dv[BQ / 32];
-#pragma unroll
-            for (int t = 0; t < BQ / 32; ++t) {
-                const int row = q0 + t * 32 + lane;
-                const bool in = row < w.q_end;
-                lv[t] = in ? __ldg(args.lse + (size_t)bh * L + row) : INFINITY;
-                dv[t] = in ? __ldg(args.delta + (size_t)bh * L + row) : 0.f;
-            }
-#pragma unroll
-            for (int t = 0; t < BQ / 32; ++t) {
-                sm.lse2[aslot][t * 32 + lane] = lv[t] * 1.4426950408889634f;
-                sm.delta[aslot][t * 32 + lane] = dv[t];
-            }
-            mbar_arrive(&sm.aux_full[aslot]);
-        }
-        STAMP(13)
-        if (lane == 0) STAMP_FLUSH(12, 14)
-    } else if (warp == MMA_WARP) {
-        // ================================================================== MMA issuer
-        // A step of 128 queries is split into two halves of 64 (a: queries 0-63, b: 64-127), each with
-        // its own S^T / dP^T columns and barriers, so that the compute warps work on one half while
-        // the tensor core produces the scores of the other half or consumes the finished one.
-        // The whole warp runs the control flow; one elected lane issues.  Descriptors are built once and
-        // advanced by adding (byte offset >> 4) to them, so issuing an MMA costs a few instructions.
-        {
+    auto get_work = [&](int g) -> BwdWork {
+        const int t = g % n_work;
+        return t < WORK_CACHE ? sm.work[t] : args.work[t];
+    };
+    auto steps_of = [](const BwdWork& w) { return (w.q_end - w.q_begin + BQ - 1) / BQ; };
+    // number of query columns of half h of step i handed to the tensor core (a multiple of 16)
+    auto half_cols = [](const BwdWork& w, int i, int h) {
+        const int n_valid = min(BQ, w.q_end - (w.q_begin + i * BQ));
+        const int n_eff = (n_valid + 15) & ~15;
+        return h == 0 ? min(n_eff, HQ) : max(n_eff - HQ, 0);
+    };
+
+    if (warp >= PRODUCER_WARP) {
+        reg_dec<REGS_MISC>();
+        if (warp == PRODUCER_WARP) {
+            // ================================================================== producer
+            // The whole warp runs the control flow; one elected lane issues the copies.
             const bool leader = elect_one();
-            STAMP_DECL
-            bool ok = __all_sync(0xffffffffu, mbar_wait(&sm.kv_full, 0, abort_flag));
-            if (!ok && lane == 0) report_timeout(args.status, 0x1200);
-            STAMP(8)
-            const uint64_t k_kd = smem_desc_sw128(smem_u32(sm.k), 16);          // K rows, K-major (A of S^T)
-            const uint64_t v_kd = smem_desc_sw128(smem_u32(sm.v), 16);          // V rows, K-major (A of dP^T)
+            if (leader) {
+                prefetch_tensormap(&map_q);
+                prefetch_tensormap(&map_k);
+                prefetch_tensormap(&map_v);
+                prefetch_tensormap(&map_do);
+            }
+            bool ok = true;
+            int gs = 0;                                     // steps issued so far, over all items
+            for (int g = item_begin; g < item_end && ok; ++g) {
+                const int bh = g / n_work;
+                const BwdWork w = get_work(g);
+                const int n_steps = steps_of(w);
+                if (g > item_begin) {
+                    // K in shared memory is read by the dQ products until the previous item is complete
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.acc_full, (g - item_begin - 1) & 1, abort_flag));
+                    if (!ok) { if (lane == 0) report_timeout(args.status, 0x1000); break; }
+                }
+                if (leader) {
+                    mbar_arrive_expect_tx(&sm.kv_full, 2 * TILE_BYTES);
+                    tma_load_3d(sm.k, &map_k, &sm.kv_full, 0, w.row_begin, bh);
+                    tma_load_3d(sm.v, &map_v, &sm.kv_full, 0, w.row_begin, bh);
+                }
+                __syncwarp();
+                for (int i = 0; i < n_steps; ++i, ++gs) {
+                    const int slot = gs % NSTAGE;
+                    const int q0 = w.q_begin + i * BQ;
+                    if (gs >= NSTAGE) {
+                        ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_empty[slot], ((gs / NSTAGE) & 1) ^ 1, abort_flag));
+                        if (!ok) { if (lane == 0) report_timeout(args.status, 0x1100 + i); break; }
+                    }
+                    if (leader) {
+                        mbar_arrive_expect_tx(&sm.qdo_full[slot], 2 * TILE_BYTES);
+                        tma_load_3d(sm.q[slot], &map_q, &sm.qdo_full[slot], 0, q0, bh);
+                        tma_load_3d(sm.dout[slot], &map_do, &sm.qdo_full[slot], 0, q0, bh);
+                    }
+                    __syncwarp();
+                }
+            }
+            if (!ok) {
+                // give the copies already issued a bounded chance to land before the block exits
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 2000000ull) { }
+            }
+        } else if (warp == AUX_WARP) {
+            // ================================================================== lse / delta loader
+            // lse and delta rows of a step go to ring slot (step count) % AUX_STAGES, several steps ahead of
+            // their use (plain loads: their row offsets are not 16-byte aligned, so TMA cannot fetch them).
+            bool ok = true;
+            int gs = 0;
+            for (int g = item_begin; g < item_end && ok; ++g) {
+                const int bh = g / n_work;
+                const BwdWork w = get_work(g);
+                const int n_steps = steps_of(w);
+                for (int i = 0; i < n_steps; ++i, ++gs) {
+                    const int aslot = gs % AUX_STAGES;
+                    if (gs >= AUX_STAGES) {
+                        ok = __all_sync(0xffffffffu,
+                                        mbar_wait(&sm.aux_empty[aslot], ((gs / AUX_STAGES) & 1) ^ 1, abort_flag));
+                        if (!ok) { if (lane == 0) report_timeout(args.status, 0x1700 + i); break; }
+                    }
+                    const int q0 = w.q_begin + i * BQ;
+                    // all loads first, then the stores: stores to shared memory in between would serialise them
+                    float lv[BQ / 32], dv[BQ / 32];
+#pragma unroll
+                    for (int t = 0; t < BQ / 32; ++t) {
+                        const int row = q0 + t * 32 + lane;
+                        const bool in = row < w.q_end;
+                        lv[t] = in ? __ldg(args.lse + (size_t)bh * L + row) : INFINITY;
+                        dv[t] = in ? __ldg(args.delta + (size_t)bh * L + row) : 0.f;
+                    }
+#pragma unroll
+                    for (int t = 0; t < BQ / 32; ++t) {
+                        sm.lse2[aslot][t * 32 + lane] = lv[t] * 1.4426950408889634f;
+                        sm.delta[aslot][t * 32 + lane] = dv[t];
+                    }
+                    mbar_arrive(&sm.aux_full[aslot]);
+                }
+            }
+        } else if (warp == MMA_WARP) {
+            // ================================================================== MMA issuer
+            // The whole warp runs the control flow and one elected lane issues (a warp that has split into
+            // one running lane and 31 parked ones issues far more slowly).  Descriptors are built once and
+            // advanced by adding (byte offset >> 4) to them.
+            // The tensor core's queue holds only a few products, and a product issued to an idle tensor core
+            // costs about a hundred clocks before it starts, so a step is issued as two uninterrupted bursts:
+            //   X_i = dV,dK of half 0 of step i, then S^T,dP^T of half 0 of step i+1
+            //   Y_i = dV,dK of half 1 of step i, dQ_i, then S^T,dP^T of half 1 of step i+1
+            // each preceded by one look at the barriers it depends on (two at a time, both usually complete).
+            const bool leader = elect_one();
             const uint64_t k_mn = smem_desc_sw128(smem_u32(sm.k), 1024);        // K as MN-major B of dQ
             // the ring slots and the dS buffers are 16 KB apart: descriptor of slot s = base + s * 1024
             const uint64_t q_kd0 = smem_desc_sw128(smem_u32(sm.q[0]), 16), do_kd0 = smem_desc_sw128(smem_u32(sm.dout[0]), 16);
             const uint64_t q_mn0 = smem_desc_sw128(smem_u32(sm.q[0]), 1024), do_mn0 = smem_desc_sw128(smem_u32(sm.dout[0]), 1024);
-            const uint64_t ds_kd0 = smem_desc_sw128(smem_u32(sm.ds[0][0]), 16);
             const uint64_t ds_mn0 = smem_desc_sw128(smem_u32(sm.ds[0][0]), TILE_BYTES);
-            constexpr uint32_t idesc_acc = idesc_bf16_f32(BKV, D, false, true);    // A K-major / TMEM, B MN-major
+            constexpr uint32_t idesc_acc = idesc_bf16_f32(BKV, D, false, true);    // A from TMEM, B MN-major
             constexpr uint32_t idesc_dq = idesc_bf16_f32(BQ, D, true, true);
-
-            auto n_eff_half = [&](int i, int h) {
-                const int n_valid = min(BQ, w.q_end - (w.q_begin + i * BQ));
-                const int n_eff = (n_valid + 15) & ~15;
-                return h == 0 ? min(n_eff, 64) : max(n_eff - 64, 0);
+            bool ok = true;
+            int gs = 0;                                         // steps issued so far (ring slot, dQ parity)
+            int ng[2] = {0, 0};                                 // gradient halves issued so far, per half
+            // waits for barrier a and, if have_b, barrier b; the two first looks overlap
+            auto wait2 = [&](uint64_t* a, uint32_t pa, uint64_t* b, uint32_t pb, bool have_b, int code) -> bool {
+                const bool ra = mbar_try_wait(a, pa);
+                const bool rb = !have_b || mbar_try_wait(b, pb);
+                if (__all_sync(0xffffffffu, ra && rb)) return true;
+                const bool done = mbar_wait(a, pa, abort_flag) && (!have_b || mbar_wait(b, pb, abort_flag));
+                if (__all_sync(0xffffffffu, done)) return true;
+                if (lane == 0) report_timeout(args.status, code);
+                return false;
             };
-            // S^T_h = K Q_h^T,  dP^T_h = V dO_h^T  for half h of step i
-            auto issue_scores = [&](int i, int h) -> bool {
-                const int slot = i % NSTAGE;
-                const int n = n_eff_half(i, h);
-                if (n == 0) return true;
-                STAMP(11)
-                if (!__all_sync(0xffffffffu, mbar_wait(&sm.qdo_full[slot], (i / NSTAGE) & 1, abort_flag))) {
-                    if (lane == 0) report_timeout(args.status, 0x1300 + i);
-                    return false;
-                }
-                STAMP(9)
-                tc_fence_after();
-                if (leader) {
-                    const uint32_t idesc = idesc_bf16_f32(BKV, n, false, false);
-                    const uint64_t qd = q_kd0 + slot * 1024 + h * 512, dd = do_kd0 + slot * 1024 + h * 512;
+            // S^T_h = K Q_h^T,  dP^T_h = V dO_h^T : n query columns of half h, Q / dO tile in ring slot `slot`
+            auto scores = [&](int h, int n, int slot) {
+                const uint32_t idesc = idesc_bf16_f32(BKV, n, false, false);
+                const uint64_t qd = q_kd0 + slot * 1024 + h * 512, dd = do_kd0 + slot * 1024 + h * 512;
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-                        mma_ss(tmem + COL_ST + h * 64, k_kd + ks * 2, qd + ks * 2, idesc, ks > 0);
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ts(tmem + COL_ST + h * HQ, tmem + COL_K + ks * 8, qd + ks * 2, idesc, ks > 0);
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks)
-                        mma_ss(tmem + COL_DPT + h * 64, v_kd + ks * 2, dd + ks * 2, idesc, ks > 0);
-                    tc_commit(&sm.s_full[h]);
-                }
-                __syncwarp();
-                return true;
+                for (int ks = 0; ks < D / 16; ++ks)
+                    mma_ts(tmem + COL_DPT + h * HQ, tmem + COL_V + ks * 8, dd + ks * 2, idesc, ks > 0);
+                tc_commit(&sm.s_full[h]);
             };
-            // dV += P_h^T dO_h,  dK += dS_h^T Q_h  for half h of step i
-            auto issue_grads = [&](int i, int h) -> bool {
-                const int slot = i % NSTAGE;
-                const int n = n_eff_half(i, h);
-                if (n == 0) return true;
-                STAMP(11)
-                if (!__all_sync(0xffffffffu, mbar_wait(&sm.p_full[h], i & 1, abort_flag))) {
-                    if (lane == 0) report_timeout(args.status, 0x1400 + i);
-                    return false;
-                }
-                STAMP(10)
-                tc_fence_after();
-                if (leader) {
-                    const int nk = n / 16;
-                    const uint64_t dod = do_mn0 + slot * 1024 + h * 512, qd = q_mn0 + slot * 1024 + h * 512;
-                    const uint64_t dsd = ds_kd0 + ((i & 1) * 2 + h) * 1024;
-                    const uint32_t p_base = tmem + COL_ST + h * 64;
-                    const bool first = (i == 0) && (h == 0);
+            // dV += P_h^T dO_h,  dK += dS_h^T Q_h : n query columns of half h
+            auto grads = [&](int h, int n, int slot, bool first) {
+                const int nk = n / 16;
+                const uint64_t dod = do_mn0 + slot * 1024 + h * 512, qd = q_mn0 + slot * 1024 + h * 512;
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        if (ks < nk)
-                            mma_ts(tmem + COL_DV, p_base + (ks / 2) * 32 + (ks % 2) * 8, dod + ks * 128, idesc_acc,
-                                   !first || (ks > 0));
+                for (int ks = 0; ks < 4; ++ks)
+                    if (ks < nk)
+                        mma_ts(tmem + COL_DV, tmem + COL_ST + h * HQ + ks * 8, dod + ks * 128, idesc_acc, !first || (ks > 0));
 #pragma unroll
-                    for (int ks = 0; ks < 4; ++ks)
-                        if (ks < nk)
-                            mma_ss(tmem + COL_DK, dsd + ks * 2, qd + ks * 128, idesc_acc, !first || (ks > 0));
-                }
-                __syncwarp();
-                return true;
+                for (int ks = 0; ks < 4; ++ks)
+                    if (ks < nk)
+                        mma_ts(tmem + COL_DK, tmem + COL_DPT + h * HQ + ks * 8, qd + ks * 128, idesc_acc, !first || (ks > 0));
             };
 
-            if (ok) ok = issue_scores(0, 0);
-            if (ok) ok = issue_scores(0, 1);
-            for (int i = 0; i < n_steps && ok; ++i) {
-                ok = issue_grads(i, 0);
-                if (ok && i + 1 < n_steps) ok = issue_scores(i + 1, 0);
-                if (ok) ok = issue_grads(i, 1);
+            for (int g = item_begin; g < item_end && ok; ++g) {
+                const BwdWork w = get_work(g);
+                const int n_steps = steps_of(w);
+                const int item = g - item_begin;
+
+                // K and V of this item are in TMEM (the compute warps copy them after the previous item's end)
+                ok = wait2(&sm.kv_tmem, item & 1, &sm.qdo_full[gs % NSTAGE], (gs / NSTAGE) & 1, true, 0x1200);
                 if (!ok) break;
-                // dQ_i = dS K over both halves: A = dS (queries x keys) read as an MN-major operand.  When
-                // the step has no second half its rows are stale data and are never drained.
+                tc_fence_after();
                 if (leader) {
-                    const uint64_t dsd = ds_mn0 + (i & 1) * 2048;
-#pragma unroll
-                    for (int ks = 0; ks < BKV / 16; ++ks)
-                        mma_ss(tmem + COL_DQ, dsd + ks * 128, k_mn + ks * 128, idesc_dq, ks > 0);
-                    tc_commit(&sm.q_empty[i % NSTAGE]);
-                    tc_commit(&sm.dq_full);
+                    scores(0, half_cols(w, 0, 0), gs % NSTAGE);
+                    const int n1 = half_cols(w, 0, 1);
+                    if (n1 > 0) scores(1, n1, gs % NSTAGE);
                 }
                 __syncwarp();
-                if (i + 1 < n_steps) ok = issue_scores(i + 1, 1);
+                // dK and dV of the previous item must have been read out before they are overwritten
+                if (item > 0) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.acc_empty, (item - 1) & 1, abort_flag));
+                    if (!ok) { if (lane == 0) report_timeout(args.status, 0x1B00); break; }
+                }
+                for (int i = 0; i < n_steps && ok; ++i, ++gs) {
+                    const int slot = gs % NSTAGE, slot_next = (gs + 1) % NSTAGE;
+                    const bool more = i + 1 < n_steps;
+                    const int n0 = half_cols(w, i, 0), n1 = half_cols(w, i, 1);
+                    const int m0 = more ? half_cols(w, i + 1, 0) : 0, m1 = more ? half_cols(w, i + 1, 1) : 0;
+                    // ---- burst X: needs P^T, dS^T of half 0 and the next step's Q / dO tile
+                    ok = wait2(&sm.p_full[0], ng[0] & 1, &sm.qdo_full[slot_next], ((gs + 1) / NSTAGE) & 1, more, 0x1400 + i);
+                    if (!ok) break;
+                    ++ng[0];
+                    tc_fence_after();
+                    if (leader) {
+                        grads(0, n0, slot, i == 0);
+                        if (m0 > 0) scores(0, m0, slot_next);
+                    }
+                    __syncwarp();
+                    // ---- burst Y: needs P^T, dS^T of half 1 (if the step has one) and dQ of the previous
+                    // step drained from TMEM
+                    if (n1 > 0) {
+                        ok = wait2(&sm.p_full[1], ng[1] & 1, &sm.dq_empty, (gs - 1) & 1, gs > 0, 0x1800 + i);
+                        ++ng[1];
+                    } else if (gs > 0) {
+                        ok = wait2(&sm.dq_empty, (gs - 1) & 1, nullptr, 0, false, 0x1800 + i);
+                    }
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (leader) {
+                        if (n1 > 0) grads(1, n1, slot, false);
+                        // dQ_i = dS K over both halves: A = dS (queries x keys) read as an MN-major operand.  When
+                        // the step has no second half its rows are stale data and are never drained.
+                        const uint64_t dsd = ds_mn0 + (gs & 1) * 2048;
+#pragma unroll
+                        for (int ks = 0; ks < BKV / 16; ++ks)
+                            mma_ss(tmem + COL_DQ, dsd + ks * 128, k_mn + ks * 128, idesc_dq, ks > 0);
+                        tc_commit(&sm.q_empty[slot]);
+                        tc_commit(&sm.dq_full);
+                        if (!more) tc_commit(&sm.acc_full);
+                        if (m1 > 0) scores(1, m1, slot_next);
+                    }
+                    __syncwarp();
+                }
             }
-            STAMP(11)
-            if (lane == 0) STAMP_FLUSH(8, 12)
         }
-    } else {
-        // ================================================================== compute warps
+    } else if (warp >= DRAIN_WARP0) {
+        // ================================================================== dQ drain
+        // One query row per thread.  dQ_i leaves TMEM 32 columns at a time, is staged in shared memory and
+        // added to the fp32 accumulator by one bulk tensor reduction per 128 x 32 piece (whole cache lines,
+        // issued by the copy engine; per-thread reductions would be 16-byte pieces of 128 different lines).
+        // Rows past the end of the query range are staged as zeros.
+        reg_dec<REGS_DRAIN>();
         const int quarter = warp & 3;
-        const int grp = warp >> 2;                          // which 32 query columns of a half
+        const int r = quarter * 32 + lane;
+        const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+        uint8_t* stage_row = sm.dq_stage + (r >> 3) * 1024 + (r & 7) * 128;
+        const bool issuer = warp == DRAIN_WARP0 && lane == 0;
+        if (issuer) prefetch_tensormap(&map_dq);
+        uint32_t buf[32];
+        bool ok = true;
+        int gs = 0;
+        uint32_t n_sync = 0;                                // meetings of the four drain warps so far
+        // all four warps meet (bounded wait, like every other wait of the kernel)
+        auto meet = [&]() -> bool {
+            mbar_arrive(&sm.drain_sync);
+            return __all_sync(0xffffffffu, mbar_wait(&sm.drain_sync, n_sync++ & 1, abort_flag));
+        };
+        for (int g = item_begin; g < item_end && ok; ++g) {
+            const int bh = g / n_work;
+            const BwdWork w = get_work(g);
+            const int n_steps = steps_of(w);
+            for (int i = 0; i < n_steps && ok; ++i, ++gs) {
+                if (!__all_sync(0xffffffffu, mbar_wait(&sm.dq_full, gs & 1, abort_flag))) {
+                    if (lane == 0) report_timeout(args.status, 0x1600 + i);
+                    ok = false;
+                    break;
+                }
+                tc_fence_after();
+                const int q0 = w.q_begin + i * BQ;
+                const bool row_in = r < min(BQ, w.q_end - q0);
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    tmem_ld32(lane_base + COL_DQ + c * 32, buf);
+                    tmem_ld_wait();
+                    if (c == 1) {
+                        tc_fence_before();
+                        mbar_arrive(&sm.dq_empty);
+                    }
+                    // the previous piece must have been read out of the staging buffer
+                    if (issuer) bulk_wait_read_all();
+                    if (!meet()) { if (lane == 0) report_timeout(args.status, 0x1C00 + i); ok = false; break; }
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) {
+                        const uint4 val = row_in ? make_uint4(buf[4 * t], buf[4 * t + 1], buf[4 * t + 2], buf[4 * t + 3])
+                                                 : make_uint4(0u, 0u, 0u, 0u);
+                        *reinterpret_cast<uint4*>(stage_row + ((t ^ (r & 7)) << 4)) = val;
+                    }
+                    fence_proxy_async_smem();
+                    if (!meet()) { if (lane == 0) report_timeout(args.status, 0x1D00 + i); ok = false; break; }
+                    if (issuer) {
+                        tma_reduce_add_2d(&map_dq, sm.dq_stage, c * 32, bh * L + q0);
+                        bulk_commit_group();
+                    }
+                }
+            }
+        }
+        if (issuer) bulk_wait_all();            // the staging buffer must outlive the last reduction's read
+    } else {
+        // ================================================================== compute warpgroups
+        reg_inc<REGS_COMPUTE>();
+        const int quarter = warp & 3;
+        const int h = warp >> 2;                            // the half of every step this warpgroup owns
         const int j = quarter * 32 + lane;                  // key row inside the tile
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
-        const bool row_ok = j < w.row_count;
-        int qlo = w.q_begin, qhi = w.q_end;                 // queries that may see this key row
-        if (!w.uniform && row_ok) {
-            const int s = scale_of_row(args.st, w.row_begin + j);
-            qlo = args.st.start[s];
-            qhi = args.st.start[min(s + 2, args.st.n_scales)];
-        }
-        const bool tile_masked = (!w.uniform) || (w.row_count < BKV);
         const float sl2 = args.scale_log2;
         const int ds_row_off = (j >> 3) * 1024 + (j & 7) * 128;
-        bool ok = true;
         uint32_t s_buf[32], dp_buf[32];
-        STAMP_DECL
+        bool ok = true;
+        int gs = 0;                                         // steps seen so far (aux ring, dS buffer parity)
+        int nsh = 0;                                        // non-empty halves of this warpgroup seen so far
 
-        // drains dQ of step `i` from TMEM into the fp32 accumulator (this thread: one query row, 32 dims)
-        auto drain_dq = [&](int i) -> bool {
-            if (!__all_sync(0xffffffffu, mbar_wait(&sm.dq_full, i & 1, abort_flag))) {
-                if (lane == 0) report_timeout(args.status, 0x1600 + i);
-                return false;
+        for (int g = item_begin; g < item_end && ok; ++g) {
+            const int bh = g / n_work;
+            const BwdWork w = get_work(g);
+            const int n_steps = steps_of(w);
+            const int item = g - item_begin;
+            const bool row_ok = j < w.row_count;
+            int qlo = w.q_begin, qhi = w.q_end;             // queries that may see this key row
+            if (!w.uniform && row_ok) {
+                const int s = scale_of_row(args.st, w.row_begin + j);
+                qlo = args.st.start[s];
+                qhi = args.st.start[min(s + 2, args.st.n_scales)];
             }
-            STAMP(3)
-            tc_fence_after();
-            const int q0 = w.q_begin + i * BQ;
-            const int n_valid = min(BQ, w.q_end - q0);
-            tmem_ld32(lane_base + COL_DQ + grp * 32, s_buf);
-            tmem_ld_wait();
-            if (j < n_valid) {
-                float* dst = args.dq_acc + ((size_t)bh * L + q0 + j) * D + grp * 32;
-#pragma unroll
-                for (int t = 0; t < 32; t += 4)
-                    red_add_v4(dst + t, __uint_as_float(s_buf[t]), __uint_as_float(s_buf[t + 1]),
-                               __uint_as_float(s_buf[t + 2]), __uint_as_float(s_buf[t + 3]));
-            }
+            const bool tile_masked = (!w.uniform) || (w.row_count < BKV);
+
+            // ---- K (warpgroup 0) / V (warpgroup 1) row to TMEM: A operands of S^T = K Q^T and dP^T = V dO^T
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.kv_full, item & 1, abort_flag));
+            if (!ok) { if (lane == 0) report_timeout(args.status, 0x1900); break; }
+            load_swizzled_row(h == 0 ? sm.k : sm.v, j, s_buf);
+            tmem_st32(lane_base + (h == 0 ? COL_K : COL_V), s_buf);
+            tmem_st_wait();
             tc_fence_before();
-            STAMP(4)
-            return true;
-        };
+            mbar_arrive(&sm.kv_tmem);
 
-        for (int i = 0; i < n_steps && ok; ++i) {
-            const int slot = i % NSTAGE;
-            const int q0 = w.q_begin + i * BQ;
-            const int n_valid = min(BQ, w.q_end - q0);
-            const int n_eff = (n_valid + 15) & ~15;
-            // visible query columns of this key row in this step: [c_lo, c_hi)
-            const int c_lo = row_ok ? max(qlo - q0, 0) : 0;
-            const int c_hi = row_ok ? min(qhi - q0, n_valid) : 0;
+            for (int i = 0; i < n_steps && ok; ++i, ++gs) {
+                const int q0 = w.q_begin + i * BQ;
+                const int n_valid = min(BQ, w.q_end - q0);
+                const int n_cols = half_cols(w, i, h);
+                const int cbase = h * HQ;                   // first query column of this half inside the step
+                // visible query columns of this key row in this step: [c_lo, c_hi)
+                const int c_lo = row_ok ? max(qlo - q0, 0) : 0;
+                const int c_hi = row_ok ? min(qhi - q0, n_valid) : 0;
 
-            const int aslot = i % AUX_STAGES;
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.aux_full[aslot], (i / AUX_STAGES) & 1, abort_flag));
-            if (!ok) { if (lane == 0) report_timeout(args.status, 0x1500 + i); break; }
-#ifdef HMAR_STAMPS
-            if (i == 0) STAMP(6) else STAMP(0)
-#endif
+                const int aslot = gs % AUX_STAGES;
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.aux_full[aslot], (gs / AUX_STAGES) & 1, abort_flag));
+                if (!ok) { if (lane == 0) report_timeout(args.status, 0x1500 + i); break; }
 
-            // dQ of the previous step must leave TMEM before this step's dQ is issued, i.e. before the
-            // last arrival of this step.  With two halves it is drained between them (the tensor core
-            // has finished it by then); a step with a single half drains it first.
-            const bool has_b = n_eff > 64;
-            if (i > 0 && !has_b) ok = drain_dq(i - 1);
-
-            for (int h = 0; h < 2 && ok; ++h) {
-                if (h == 1 && !has_b) break;
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[h], i & 1, abort_flag));
-                if (!ok) { if (lane == 0) report_timeout(args.status, 0x1580 + i); break; }
-                STAMP(1)
-                tc_fence_after();
-                const int c0 = h * 64 + grp * 32;           // first query column of this thread's chunk
-                if (c0 < n_eff) {
-                    tmem_ld32(lane_base + COL_ST + c0, s_buf);
-                    tmem_ld32(lane_base + COL_DPT + c0, dp_buf);
-                    // lse / delta of the chunk's 32 queries while the TMEM loads are in flight
-                    float4 ls[8], de[8];
-                    const float4* lse4 = reinterpret_cast<const float4*>(&sm.lse2[aslot][c0]);
-                    const float4* del4 = reinterpret_cast<const float4*>(&sm.delta[aslot][c0]);
+                if (n_cols > 0) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[h], nsh & 1, abort_flag));
+                    if (!ok) { if (lane == 0) report_timeout(args.status, 0x1580 + i); break; }
+                    ++nsh;
+                    tc_fence_after();
+                    uint8_t* ds_row = sm.ds[gs & 1][h] + ds_row_off;
 #pragma unroll
-                    for (int t = 0; t < 8; ++t) { ls[t] = lse4[t]; de[t] = del4[t]; }
-                    tmem_ld_wait();
-                    STAMP(14)
-                    uint32_t p_pack[16], ds_pack[16];
+                    for (int c = 0; c < 2; ++c) {           // 32 query columns at a time
+                        if (c * 32 < n_cols) {
+                            const int c0 = cbase + c * 32;  // first query column of the chunk inside the step
+                            tmem_ld32(lane_base + COL_ST + c0, s_buf);
+                            tmem_ld32(lane_base + COL_DPT + c0, dp_buf);
+                            // lse / delta of the chunk's 32 queries while the TMEM loads are in flight
+                            float4 ls[8], de[8];
+                            const float4* lse4 = reinterpret_cast<const float4*>(&sm.lse2[aslot][c0]);
+                            const float4* del4 = reinterpret_cast<const float4*>(&sm.delta[aslot][c0]);
 #pragma unroll
-                    for (int t = 0; t < 32; t += 4) {
-                        float p0 = ex2(fmaf(__uint_as_float(s_buf[t]), sl2, -ls[t / 4].x));
-                        float p1 = ex2(fmaf(__uint_as_float(s_buf[t + 1]), sl2, -ls[t / 4].y));
-                        float p2 = ex2(fmaf(__uint_as_float(s_buf[t + 2]), sl2, -ls[t / 4].z));
-                        float p3 = ex2(fmaf(__uint_as_float(s_buf[t + 3]), sl2, -ls[t / 4].w));
-                        if (tile_masked) {
-                            p0 = (c0 + t >= c_lo && c0 + t < c_hi) ? p0 : 0.f;
-                            p1 = (c0 + t + 1 >= c_lo && c0 + t + 1 < c_hi) ? p1 : 0.f;
-                            p2 = (c0 + t + 2 >= c_lo && c0 + t + 2 < c_hi) ? p2 : 0.f;
-                            p3 = (c0 + t + 3 >= c_lo && c0 + t + 3 < c_hi) ? p3 : 0.f;
+                            for (int t = 0; t < 8; ++t) { ls[t] = lse4[t]; de[t] = del4[t]; }
+                            tmem_ld_wait();
+                            uint32_t p_pack[16], ds_pack[16];
+#pragma unroll
+                            for (int t = 0; t < 32; t += 4) {
+                                float p0 = ex2(fmaf(__uint_as_float(s_buf[t]), sl2, -ls[t / 4].x));
+                                float p1 = ex2(fmaf(__uint_as_float(s_buf[t + 1]), sl2, -ls[t / 4].y));
+                                float p2 = ex2(fmaf(__uint_as_float(s_buf[t + 2]), sl2, -ls[t / 4].z));
+                                float p3 = ex2(fmaf(__uint_as_float(s_buf[t + 3]), sl2, -ls[t / 4].w));
+                                if (tile_masked) {
+                                    p0 = (c0 + t >= c_lo && c0 + t < c_hi) ? p0 : 0.f;
+                                    p1 = (c0 + t + 1 >= c_lo && c0 + t + 1 < c_hi) ? p1 : 0.f;
+                                    p2 = (c0 + t + 2 >= c_lo && c0 + t + 2 < c_hi) ? p2 : 0.f;
+                                    p3 = (c0 + t + 3 >= c_lo && c0 + t + 3 < c_hi) ? p3 : 0.f;
+                                }
+                                const float d0 = p0 * (__uint_as_float(dp_buf[t]) - de[t / 4].x);
+                                const float d1 = p1 * (__uint_as_float(dp_buf[t + 1]) - de[t / 4].y);
+                                const float d2 = p2 * (__uint_as_float(dp_buf[t + 2]) - de[t / 4].z);
+                                const float d3 = p3 * (__uint_as_float(dp_buf[t + 3]) - de[t / 4].w);
+                                p_pack[t / 2] = pack_bf16(p0, p1);
+                                p_pack[t / 2 + 1] = pack_bf16(p2, p3);
+                                ds_pack[t / 2] = pack_bf16(d0, d1);
+                                ds_pack[t / 2 + 1] = pack_bf16(d2, d3);
+                            }
+                            // P^T over S^T and dS^T over dP^T: the 16 packed columns of chunk c start at column
+                            // c * 16 of the half, which this thread has already read
+                            tmem_st16(lane_base + COL_ST + cbase + c * 16, p_pack);
+                            tmem_st16(lane_base + COL_DPT + cbase + c * 16, ds_pack);
+                            // dS^T to shared memory: 4 pieces of 8 queries, 128-byte swizzle on the key row
+#pragma unroll
+                            for (int ch = 0; ch < 4; ++ch) {
+                                const int piece = c * 4 + ch;
+                                uint4 val = make_uint4(ds_pack[4 * ch], ds_pack[4 * ch + 1], ds_pack[4 * ch + 2], ds_pack[4 * ch + 3]);
+                                *reinterpret_cast<uint4*>(ds_row + ((piece ^ (j & 7)) << 4)) = val;
+                            }
                         }
-                        const float d0 = p0 * (__uint_as_float(dp_buf[t]) - de[t / 4].x);
-                        const float d1 = p1 * (__uint_as_float(dp_buf[t + 1]) - de[t / 4].y);
-                        const float d2 = p2 * (__uint_as_float(dp_buf[t + 2]) - de[t / 4].z);
-                        const float d3 = p3 * (__uint_as_float(dp_buf[t + 3]) - de[t / 4].w);
-                        p_pack[t / 2] = pack_bf16(p0, p1);
-                        p_pack[t / 2 + 1] = pack_bf16(p2, p3);
-                        ds_pack[t / 2] = pack_bf16(d0, d1);
-                        ds_pack[t / 2 + 1] = pack_bf16(d2, d3);
-                    }
-                    STAMP(15)
-                    // P^T over S^T: the 16 packed columns written here start at this thread's own first
-                    // fp32 column, which it has already read
-                    tmem_st16(lane_base + COL_ST + c0, p_pack);
-                    // dS^T to shared memory: 4 chunks of 8 queries, 128-byte swizzle on the key row
-                    uint8_t* ds_row = sm.ds[i & 1][h] + ds_row_off;
-#pragma unroll
-                    for (int ch = 0; ch < 4; ++ch) {
-                        const int chunk = grp * 4 + ch;
-                        uint4 val = make_uint4(ds_pack[4 * ch], ds_pack[4 * ch + 1], ds_pack[4 * ch + 2], ds_pack[4 * ch + 3]);
-                        *reinterpret_cast<uint4*>(ds_row + ((chunk ^ (j & 7)) << 4)) = val;
                     }
                     tmem_st_wait();
+                    tc_fence_before();
+                    fence_proxy_async_smem();
+                    mbar_arrive(&sm.p_full[h]);
                 }
-                tc_fence_before();
-                fence_proxy_async_smem();
-                mbar_arrive(&sm.p_full[h]);
-                STAMP(2)
-                if (h == 0 && i > 0 && has_b) ok = drain_dq(i - 1);
+                mbar_arrive(&sm.aux_empty[aslot]);      // this thread is done with the step's lse / delta
             }
-            mbar_arrive(&sm.aux_empty[aslot]);      // this thread is done with the step's lse / delta
-        }
-        if (ok) ok = drain_dq(n_steps - 1);
-        const int half = grp;
+            if (!ok) break;
 
-        // ---- epilogue: dK (warps 0-3) and dV (warps 4-7); the last dq_full also covers them
-        if (ok) {
-            const uint32_t col = half == 0 ? COL_DK : COL_DV;
-            const float mul = half == 0 ? args.softmax_scale : 1.f;
-            __nv_bfloat16* base = half == 0 ? args.dk : args.dv;
-            __nv_bfloat16* orow = base + ((size_t)bh * L + w.row_begin + j) * D;
+            // ---- end of the item: dK (warpgroup 0) and dV (warpgroup 1), one key row per thread
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.acc_full, item & 1, abort_flag));
+            if (!ok) { if (lane == 0) report_timeout(args.status, 0x1A00); break; }
+            tc_fence_after();
+            tmem_ld32(lane_base + (h == 0 ? COL_DK : COL_DV), s_buf);
+            tmem_ld32(lane_base + (h == 0 ? COL_DK : COL_DV) + 32, dp_buf);
+            tmem_ld_wait();
+            tc_fence_before();
+            mbar_arrive(&sm.acc_empty);                 // the next item's products may overwrite dK / dV
+            if (row_ok) {
+                const float mul = h == 0 ? args.softmax_scale : 1.f;
+                __nv_bfloat16* base = h == 0 ? args.dk : args.dv;
+                uint4* dst = reinterpret_cast<uint4*>(base + ((size_t)bh * L + w.row_begin + j) * D);
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                tmem_ld32(lane_base + col + h * 32, s_buf);
-                tmem_ld_wait();
-                if (row_ok) {
-                    uint4* dst = reinterpret_cast<uint4*>(orow + h * 32);
+                for (int t = 0; t < 4; ++t) {
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(s_buf[8 * t + 0]) * mul, __uint_as_float(s_buf[8 * t + 1]) * mul);
+                    o.y = pack_bf16(__uint_as_float(s_buf[8 * t + 2]) * mul, __uint_as_float(s_buf[8 * t + 3]) * mul);
+                    o.z = pack_bf16(__uint_as_float(s_buf[8 * t + 4]) * mul, __uint_as_float(s_buf[8 * t + 5]) * mul);
+                    o.w = pack_bf16(__uint_as_float(s_buf[8 * t + 6]) * mul, __uint_as_float(s_buf[8 * t + 7]) * mul);
+                    dst[t] = o;
+                }
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        uint4 o;
-                        o.x = pack_bf16(__uint_as_float(s_buf[8 * t + 0]) * mul, __uint_as_float(s_buf[8 * t + 1]) * mul);
-                        o.y = pack_bf16(__uint_as_float(s_buf[8 * t + 2]) * mul, __uint_as_float(s_buf[8 * t + 3]) * mul);
-                        o.z = pack_bf16(__uint_as_float(s_buf[8 * t + 4]) * mul, __uint_as_float(s_buf[8 * t + 5]) * mul);
-                        o.w = pack_bf16(__uint_as_float(s_buf[8 * t + 6]) * mul, __uint_as_float(s_buf[8 * t + 7]) * mul);
-                        dst[t] = o;
-                    }
+                for (int t = 0; t < 4; ++t) {
+                    uint4 o;
+                    o.x = pack_bf16(__uint_as_float(dp_buf[8 * t + 0]) * mul, __uint_as_float(dp_buf[8 * t + 1]) * mul);
+                    o.y = pack_bf16(__uint_as_float(dp_buf[8 * t + 2]) * mul, __uint_as_float(dp_buf[8 * t + 3]) * mul);
+                    o.z = pack_bf16(__uint_as_float(dp_buf[8 * t + 4]) * mul, __uint_as_float(dp_buf[8 * t + 5]) * mul);
+                    o.w = pack_bf16(__uint_as_float(dp_buf[8 * t + 6]) * mul, __uint_as_float(dp_buf[8 * t + 7]) * mul);
+                    dst[4 + t] = o;
                 }
             }
         }
-        STAMP(5)
-        if (warp == 0 && lane == 0) { STAMP_FLUSH(0, 7) STAMP_FLUSH(14, 16) }
     }
 
     tc_fence_before();
@@ -474,18 +620,6 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         tmem_dealloc(tmem, TMEM_COLS);
     }
 }
-
-#ifdef HMAR_STAMPS
-}  // namespace
-extern "C" int hmar_debug_bwd_stamps(unsigned long long* out16) {
-    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
-    if (cudaMemcpyFromSymbol(out16, g_bwd_stamps, sizeof(g_bwd_stamps)) != cudaSuccess) return -1;
-    unsigned long long zero[16] = {0};
-    cudaMemcpyToSymbol(g_bwd_stamps, zero, sizeof(zero));
-    return 0;
-}
-namespace {
-#endif
 
 // ------------------------------------------------------------------------------------------------
 // delta_i = sum_d dO_id * O_id  (one warp per 4 rows: 8 lanes x 16 bytes cover a row)
@@ -530,8 +664,21 @@ hmar_bwd_dq_convert_kernel(const float* __restrict__ acc, __nv_bfloat16* __restr
 
 }  // namespace
 
+// Number of SMs of the current device (one persistent block each), looked up once per device.
+static int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 1;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& dout_map,
-                          const BwdArgs& args, const __nv_bfloat16* out, const __nv_bfloat16* dout,
+                          const CUtensorMap& dq_acc_map, const BwdArgs& args, const __nv_bfloat16* out, const __nv_bfloat16* dout,
                           __nv_bfloat16* dq, int BH, cudaStream_t stream) {
     const size_t smem = sizeof(SharedStorage) + 1024;
     cudaError_t e = cudaFuncSetAttribute(hmar_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -548,7 +695,9 @@ cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUte
     }
     {
         KernelTimer timer("hmar_bwd_tc_kernel", stream);
-        hmar_bwd_tc_kernel<<<(unsigned)BH * (unsigned)args.n_work, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, args);
+        const long long items = (long long)BH * args.n_work;
+        const unsigned grid = (unsigned)(items < sm_count() ? items : sm_count());
+        hmar_bwd_tc_kernel<<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, args);
     }
     const size_t n8 = n_rows * D / 8;
     {

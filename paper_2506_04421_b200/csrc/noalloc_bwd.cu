@@ -52,6 +52,7 @@ static unsigned char* scratch_address() {
 }
 
 bool make_rows_map_bf16(CUtensorMap* map, const void* base, int heads, int rows);
+bool make_dq_acc_map(CUtensorMap* map, const float* base, size_t rows);
 
 }  // namespace hmar
 
@@ -99,6 +100,7 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
         host_work[i].q_end = tiles[i].partner_end;
         host_work[i].uniform = tiles[i].uniform;
     }
+    const int head_cost = bwd_fill_costs(host_work, (int)tiles.size());
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // Pageable source: the runtime stages it before returning, so the stack buffer may go away.
     if (cudaMemcpyAsync(scratch, host_work, tiles.size() * sizeof(BwdWork), cudaMemcpyHostToDevice, s) != cudaSuccess) {
@@ -107,13 +109,16 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
     }
 
     const int BH = B * H;
-    CUtensorMap mq, mk, mv, mdo;
+    CUtensorMap mq, mk, mv, mdo, macc;
     if (!make_rows_map_bf16(&mq, q, BH, (int)L) || !make_rows_map_bf16(&mk, k, BH, (int)L) ||
-        !make_rows_map_bf16(&mv, v, BH, (int)L) || !make_rows_map_bf16(&mdo, dout, BH, (int)L))
+        !make_rows_map_bf16(&mv, v, BH, (int)L) || !make_rows_map_bf16(&mdo, dout, BH, (int)L) ||
+        !make_dq_acc_map(&macc, reinterpret_cast<const float*>(scratch + kWorkBytes + kDeltaBytes), (size_t)BH * L))
         return HMAR_ERR_CUDA;
     BwdArgs a{};
     a.work = reinterpret_cast<const BwdWork*>(scratch);
     a.n_work = (int)tiles.size();
+    a.n_heads = BH;
+    a.head_cost = head_cost;
     a.L = (int)L;
     a.scale_log2 = softmax_scale * 1.4426950408889634f;
     a.softmax_scale = softmax_scale;
@@ -125,7 +130,7 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
     a.dv = static_cast<__nv_bfloat16*>(dv);
     a.status = nullptr;
     a.st = st;
-    return launch_bwd_tc(mq, mk, mv, mdo, a, static_cast<const __nv_bfloat16*>(out),
+    return launch_bwd_tc(mq, mk, mv, mdo, macc, a, static_cast<const __nv_bfloat16*>(out),
                          static_cast<const __nv_bfloat16*>(dout), static_cast<__nv_bfloat16*>(dq), BH, s) == cudaSuccess
                ? HMAR_OK : HMAR_ERR_CUDA;
 }

@@ -34,12 +34,26 @@ struct BwdWork {
     int32_t row_begin, row_count;
     int32_t q_begin, q_end;
     int32_t uniform;
-    int32_t pad[3];
+    int32_t cost_begin;      // cost of the head's tiles before this one (see bwd_fill_costs)
+    int32_t pad[2];
 };
+
+// Cost model of the backward's persistent blocks: a tile costs its number of 128-query steps plus a
+// constant for the work at its start and end.  Fills cost_begin and returns the cost of a whole head.
+inline int bwd_fill_costs(BwdWork* work, int n) {
+    int acc = 0;
+    for (int i = 0; i < n; ++i) {
+        work[i].cost_begin = acc;
+        acc += (work[i].q_end - work[i].q_begin + 127) / 128 + 2;
+    }
+    return acc;
+}
 
 struct BwdArgs {
     const BwdWork* work;
     int n_work;
+    int n_heads;             // B * H
+    int head_cost;           // from bwd_fill_costs
     int L;
     float scale_log2;        // softmax_scale * log2(e)
     float softmax_scale;
@@ -55,7 +69,7 @@ struct BwdArgs {
 
 size_t fwd_tc_smem_bytes();
 cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& dout_map,
-                          const BwdArgs& args, const __nv_bfloat16* out, const __nv_bfloat16* dout,
+                          const CUtensorMap& dq_acc_map, const BwdArgs& args, const __nv_bfloat16* out, const __nv_bfloat16* dout,
                           __nv_bfloat16* dq, int BH, cudaStream_t stream);
 cudaError_t launch_fwd_tc(const CUtensorMap& q, const CUtensorMap& k0, const CUtensorMap& v0, const CUtensorMap& k1,
                           const CUtensorMap& v1, const FwdArgs& args, int BH, cudaStream_t stream);

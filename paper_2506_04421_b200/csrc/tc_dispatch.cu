@@ -51,6 +51,20 @@ static bool make_rows_map(CUtensorMap* map, const void* base, int heads, int row
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of the fp32 dQ accumulator seen as [rows, 64]: boxes of 128 rows x 32 columns (128 bytes,
+// 128-byte swizzle), the unit in which the backward kernel adds dQ tiles to it.
+static bool make_acc_map(CUtensorMap* map, const float* base, size_t rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 4};
+    const cuuint32_t box[2] = {32, (cuuint32_t)kTileRows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Plan cache: one entry per (device, side length list).
 struct Plan {
@@ -58,6 +72,7 @@ struct Plan {
     BwdWork* bwd_work = nullptr;
     int n_fwd = 0;
     int n_bwd = 0;
+    int bwd_head_cost = 0;
 };
 
 struct PlanKey {
@@ -102,6 +117,7 @@ static const Plan* get_plan(const ScaleTable& st) {
     }
     static_assert(sizeof(FwdWork) == sizeof(BwdWork), "work tiles share one allocation");
     Plan plan;
+    plan.bwd_head_cost = bwd_fill_costs(bwork.data(), (int)bwork.size());
     plan.n_fwd = (int)work.size();
     plan.n_bwd = (int)bwork.size();
     const size_t fwd_bytes = work.size() * sizeof(FwdWork), bwd_bytes = bwork.size() * sizeof(BwdWork);
@@ -192,13 +208,15 @@ int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const f
     const Plan* plan = get_plan(st);
     if (plan == nullptr) return HMAR_ERR_CUDA;
     const int L = st.start[st.n_scales];
-    CUtensorMap mq, mk, mv, mdo;
+    CUtensorMap mq, mk, mv, mdo, macc;
     if (!make_rows_map(&mq, q, BH, L) || !make_rows_map(&mk, k, BH, L) || !make_rows_map(&mv, v, BH, L) ||
-        !make_rows_map(&mdo, dout, BH, L))
+        !make_rows_map(&mdo, dout, BH, L) || !make_acc_map(&macc, dq_acc, (size_t)BH * L))
         return HMAR_ERR_CUDA;
     BwdArgs a{};
     a.work = plan->bwd_work;
     a.n_work = plan->n_bwd;
+    a.n_heads = BH;
+    a.head_cost = plan->bwd_head_cost;
     a.L = L;
     a.scale_log2 = scale * 1.4426950408889634f;
     a.softmax_scale = scale;
@@ -210,12 +228,13 @@ int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const f
     a.dv = dv;
     a.status = status;
     a.st = st;
-    return launch_bwd_tc(mq, mk, mv, mdo, a, out, dout, dq, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
+    return launch_bwd_tc(mq, mk, mv, mdo, macc, a, out, dout, dq, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
-// Same tensor map as above for code outside this file.
+// The same tensor maps for code outside this file.
 bool make_rows_map_bf16(CUtensorMap* map, const void* base, int heads, int rows) {
     return make_rows_map(map, base, heads, rows);
 }
+bool make_dq_acc_map(CUtensorMap* map, const float* base, size_t rows) { return make_acc_map(map, base, rows); }
 
 }  // namespace hmar
