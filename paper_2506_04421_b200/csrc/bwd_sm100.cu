@@ -69,13 +69,13 @@ struct __align__(1024) SharedStorage {
     uint8_t q[NSTAGE][TILE_BYTES];
     uint8_t dout[NSTAGE][TILE_BYTES];
     uint8_t ds[2][2][TILE_BYTES];           // dS^T, double buffered: [step parity][64-query half][key row][64 queries], 128B swizzle
-    uint8_t dq_stage[TILE_BYTES];           // 128 query rows x 32 fp32 columns of dQ_i on their way to the accumulator, 128B swizzle
+    uint8_t dq_stage[TILE_BYTES];           // per drain warp: 32 query rows x 32 fp32 columns of dQ_i on their way to the accumulator, 128B swizzle
     float lse2[AUX_STAGES][BQ];             // lse * log2(e); +inf for query rows outside the range
     float delta[AUX_STAGES][BQ];
     uint64_t kv_full, kv_tmem;
     uint64_t qdo_full[NSTAGE], q_empty[NSTAGE], aux_full[AUX_STAGES], aux_empty[AUX_STAGES];
     uint64_t s_full[2], p_full[2];            // [half of the step]
-    uint64_t dq_full, dq_empty, acc_full, acc_empty, drain_sync;
+    uint64_t dq_full, dq_empty, acc_full, acc_empty;
     BwdWork work[WORK_CACHE];               // the head's work list (its first WORK_CACHE tiles)
     uint32_t tmem_base;
     int abort_flag;
@@ -93,7 +93,7 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// Adds a [128 rows x 32 fp32] tile in shared memory (128-byte swizzle) to global memory at (column c0, row c1).
+// Adds a [32 rows x 32 fp32] tile in shared memory (128-byte swizzle) to global memory at (column c0, row c1).
 __device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* m, const void* smem_src, int c0, int c1) {
     asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
                  ::"l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(smem_src)), "r"(c0), "r"(c1)
@@ -169,7 +169,6 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         mbar_init(&sm.dq_empty, 128);
         mbar_init(&sm.acc_full, 1);
         mbar_init(&sm.acc_empty, NUM_COMPUTE_THREADS);
-        mbar_init(&sm.drain_sync, 128);
         fence_mbar_init();
         const long long total = (long long)args.n_heads * args.head_cost;
         sm.item_begin = first_item_at_cost(args, total * blockIdx.x / gridDim.x);
@@ -292,7 +291,7 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // The tensor core's queue holds only a few products, and a product issued to an idle tensor core
             // costs about a hundred clocks before it starts, so a step is issued as two uninterrupted bursts:
             //   X_i = dV,dK of half 0 of step i, then S^T,dP^T of half 0 of step i+1
-            //   Y_i = dV,dK of half 1 of step i, dQ_i, then S^T,dP^T of half 1 of step i+1
+            //   Y_i = dV,dK of half 1 of step i, then S^T,dP^T of half 1 of step i+1, then dQ_i
             // each preceded by one look at the barriers it depends on (two at a time, both usually complete).
             const bool leader = elect_one();
             const uint64_t k_mn = smem_desc_sw128(smem_u32(sm.k), 1024);        // K as MN-major B of dQ
@@ -388,16 +387,18 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     tc_fence_after();
                     if (leader) {
                         if (n1 > 0) grads(1, n1, slot, false);
+                        tc_commit(&sm.q_empty[slot]);           // Q_i, dO_i are not read again
+                        // the next scores of half 1 go first: the compute warpgroup is waiting for them, dQ_i
+                        // is not needed before the drain warps get to it
+                        if (m1 > 0) scores(1, m1, slot_next);
                         // dQ_i = dS K over both halves: A = dS (queries x keys) read as an MN-major operand.  When
                         // the step has no second half its rows are stale data and are never drained.
                         const uint64_t dsd = ds_mn0 + (gs & 1) * 2048;
 #pragma unroll
                         for (int ks = 0; ks < BKV / 16; ++ks)
                             mma_ss(tmem + COL_DQ, dsd + ks * 128, k_mn + ks * 128, idesc_dq, ks > 0);
-                        tc_commit(&sm.q_empty[slot]);
                         tc_commit(&sm.dq_full);
                         if (!more) tc_commit(&sm.acc_full);
-                        if (m1 > 0) scores(1, m1, slot_next);
                     }
                     __syncwarp();
                 }
@@ -405,31 +406,26 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
     } else if (warp >= DRAIN_WARP0) {
         // ================================================================== dQ drain
-        // One query row per thread.  dQ_i leaves TMEM 32 columns at a time, is staged in shared memory and
-        // added to the fp32 accumulator by one bulk tensor reduction per 128 x 32 piece (whole cache lines,
-        // issued by the copy engine; per-thread reductions would be 16-byte pieces of 128 different lines).
-        // Rows past the end of the query range are staged as zeros.
+        // One query row per thread, and every warp on its own: dQ_i leaves TMEM 32 columns at a time, is
+        // staged in the warp's 4 KB of shared memory and added to the fp32 accumulator by one bulk tensor
+        // reduction per 32 x 32 piece (whole cache lines, issued by the copy engine; per-thread reductions
+        // would be 16-byte pieces of 32 different lines).  Rows past the end of the query range are staged
+        // as zeros.
         reg_dec<REGS_DRAIN>();
         const int quarter = warp & 3;
         const int r = quarter * 32 + lane;
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
-        uint8_t* stage_row = sm.dq_stage + (r >> 3) * 1024 + (r & 7) * 128;
-        const bool issuer = warp == DRAIN_WARP0 && lane == 0;
-        if (issuer) prefetch_tensormap(&map_dq);
+        uint8_t* stage = sm.dq_stage + quarter * 4096;
+        uint8_t* stage_row = stage + (lane >> 3) * 1024 + (lane & 7) * 128;
+        if (lane == 0) prefetch_tensormap(&map_dq);
         uint32_t buf[32];
         bool ok = true;
         int gs = 0;
-        uint32_t n_sync = 0;                                // meetings of the four drain warps so far
-        // all four warps meet (bounded wait, like every other wait of the kernel)
-        auto meet = [&]() -> bool {
-            mbar_arrive(&sm.drain_sync);
-            return __all_sync(0xffffffffu, mbar_wait(&sm.drain_sync, n_sync++ & 1, abort_flag));
-        };
         for (int g = item_begin; g < item_end && ok; ++g) {
             const int bh = g / n_work;
             const BwdWork w = get_work(g);
             const int n_steps = steps_of(w);
-            for (int i = 0; i < n_steps && ok; ++i, ++gs) {
+            for (int i = 0; i < n_steps; ++i, ++gs) {
                 if (!__all_sync(0xffffffffu, mbar_wait(&sm.dq_full, gs & 1, abort_flag))) {
                     if (lane == 0) report_timeout(args.status, 0x1600 + i);
                     ok = false;
@@ -447,24 +443,24 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         mbar_arrive(&sm.dq_empty);
                     }
                     // the previous piece must have been read out of the staging buffer
-                    if (issuer) bulk_wait_read_all();
-                    if (!meet()) { if (lane == 0) report_timeout(args.status, 0x1C00 + i); ok = false; break; }
+                    if (lane == 0) bulk_wait_read_all();
+                    __syncwarp();
 #pragma unroll
                     for (int t = 0; t < 8; ++t) {
                         const uint4 val = row_in ? make_uint4(buf[4 * t], buf[4 * t + 1], buf[4 * t + 2], buf[4 * t + 3])
                                                  : make_uint4(0u, 0u, 0u, 0u);
-                        *reinterpret_cast<uint4*>(stage_row + ((t ^ (r & 7)) << 4)) = val;
+                        *reinterpret_cast<uint4*>(stage_row + ((t ^ (lane & 7)) << 4)) = val;
                     }
                     fence_proxy_async_smem();
-                    if (!meet()) { if (lane == 0) report_timeout(args.status, 0x1D00 + i); ok = false; break; }
-                    if (issuer) {
-                        tma_reduce_add_2d(&map_dq, sm.dq_stage, c * 32, bh * L + q0);
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_reduce_add_2d(&map_dq, stage, c * 32, bh * L + q0 + quarter * 32);
                         bulk_commit_group();
                     }
                 }
             }
         }
-        if (issuer) bulk_wait_all();            // the staging buffer must outlive the last reduction's read
+        if (lane == 0) bulk_wait_all();         // the staging buffer must outlive the last reduction's read
     } else {
         // ================================================================== compute warpgroups
         reg_inc<REGS_COMPUTE>();

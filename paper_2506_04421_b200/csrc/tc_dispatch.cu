@@ -51,14 +51,14 @@ static bool make_rows_map(CUtensorMap* map, const void* base, int heads, int row
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tensor map of the fp32 dQ accumulator seen as [rows, 64]: boxes of 128 rows x 32 columns (128 bytes,
-// 128-byte swizzle), the unit in which the backward kernel adds dQ tiles to it.
+// Tensor map of the fp32 dQ accumulator seen as [rows, 64]: boxes of 32 rows x 32 columns (128 bytes,
+// 128-byte swizzle), the unit in which a warp of the backward kernel adds dQ pieces to it.
 static bool make_acc_map(CUtensorMap* map, const float* base, size_t rows) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)kHeadDim * 4};
-    const cuuint32_t box[2] = {32, (cuuint32_t)kTileRows};
+    const cuuint32_t box[2] = {32, 32};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
