@@ -54,9 +54,9 @@ constexpr int NUM_COMPUTE_THREADS = 256;
 constexpr int DRAIN_WARP0 = 8, PRODUCER_WARP = 12, MMA_WARP = 13, AUX_WARP = 14;
 constexpr int NUM_THREADS = 512;
 #ifndef X_RC
-#define X_RC 176
-#define X_RD 64
-#define X_RM 96
+#define X_RC 160
+#define X_RD 72
+#define X_RM 120
 #endif
 constexpr int REGS_COMPUTE = X_RC, REGS_DRAIN = X_RD, REGS_MISC = X_RM;
 static_assert(2 * REGS_COMPUTE + REGS_DRAIN + REGS_MISC == 4 * 128, "register budget of the block");
