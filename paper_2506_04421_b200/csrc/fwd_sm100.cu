@@ -142,31 +142,41 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
     if (warp == 0) {
         // ================================================================== TMA producer
-        if (lane == 0) {
+        // The whole warp runs the control flow; one elected lane issues the copies (a warp that has split
+        // into one running lane and 31 parked ones issues far more slowly).
+        const bool leader = elect_one();
+        if (leader) {
             prefetch_tensormap(&map_q);
             prefetch_tensormap(&map_k0);
             prefetch_tensormap(&map_v0);
             mbar_arrive_expect_tx(&sm.q_full, TILE_BYTES);
             tma_load_3d(sm.q, &map_q, &sm.q_full, 0, w.row_begin, bh);
-            bool ok = true;
-            for (int j = 0; j < n_tiles && ok; ++j) {
-                const int slot = j % NSTAGE;
-                const uint32_t par = ((j / NSTAGE) & 1) ^ 1;     // parity of the previous use of the slot
-                const KvTile t = kv_tile(w, tiles0, j);
-                if (j >= NSTAGE) ok = mbar_wait(&sm.k_empty[slot], par, abort_flag);
-                if (!ok) { report_timeout(args.status, 0x100 + j); break; }
+        }
+        __syncwarp();
+        bool ok = true;
+        for (int j = 0; j < n_tiles && ok; ++j) {
+            const int slot = j % NSTAGE;
+            const uint32_t par = ((j / NSTAGE) & 1) ^ 1;     // parity of the previous use of the slot
+            const KvTile t = kv_tile(w, tiles0, j);
+            if (j >= NSTAGE) ok = __all_sync(0xffffffffu, mbar_wait(&sm.k_empty[slot], par, abort_flag));
+            if (!ok) { if (lane == 0) report_timeout(args.status, 0x100 + j); break; }
+            if (leader) {
                 mbar_arrive_expect_tx(&sm.k_full[slot], TILE_BYTES);
                 tma_load_3d(sm.k[slot], t.seg ? &map_k1 : &map_k0, &sm.k_full[slot], 0, t.coord, bh);
-                if (j >= NSTAGE) ok = mbar_wait(&sm.v_empty[slot], par, abort_flag);
-                if (!ok) { report_timeout(args.status, 0x200 + j); break; }
+            }
+            __syncwarp();
+            if (j >= NSTAGE) ok = __all_sync(0xffffffffu, mbar_wait(&sm.v_empty[slot], par, abort_flag));
+            if (!ok) { if (lane == 0) report_timeout(args.status, 0x200 + j); break; }
+            if (leader) {
                 mbar_arrive_expect_tx(&sm.v_full[slot], TILE_BYTES);
                 tma_load_3d(sm.v[slot], t.seg ? &map_v1 : &map_v0, &sm.v_full[slot], 0, t.coord, bh);
             }
-            if (!ok) {
-                // give the copies already issued a bounded chance to land before the block exits
-                const uint64_t t0 = globaltimer_ns();
-                while (globaltimer_ns() - t0 < 2000000ull) { }
-            }
+            __syncwarp();
+        }
+        if (!ok) {
+            // give the copies already issued a bounded chance to land before the block exits
+            const uint64_t t0 = globaltimer_ns();
+            while (globaltimer_ns() - t0 < 2000000ull) { }
         }
     } else if (warp == 1) {
         // ================================================================== MMA issuer
