@@ -120,6 +120,57 @@ __device__ __forceinline__ void load_swizzled_row(const uint8_t* tile, int r, ui
     }
 }
 
+// One key row, 32 query columns (chunk c of the half that starts at column cbase of the step):
+// P^T = 2^(S^T * scale * log2e - lse * log2e) and dS^T = P^T o (dP^T - delta) in fp32.  P^T (bf16) goes back to
+// TMEM over S^T and dS^T (bf16) over dP^T - the 16 packed columns of chunk c start at column c * 16 of the
+// half, which this thread has already read - and dS^T also goes to shared memory (4 pieces of 8 queries,
+// 128-byte swizzle on the key row j).  MASKED: only columns [c_lo, c_hi) of the step are visible to this row.
+template <bool MASKED>
+__device__ __forceinline__ void softmax_grad_chunk(uint32_t lane_base, int cbase, int c, const float* lse2, const float* delta,
+                                                   float sl2, int c_lo, int c_hi, uint8_t* ds_row, int j) {
+    const int c0 = cbase + c * 32;          // first query column of the chunk inside the step
+    uint32_t s_buf[32], dp_buf[32];
+    tmem_ld32(lane_base + COL_ST + c0, s_buf);
+    tmem_ld32(lane_base + COL_DPT + c0, dp_buf);
+    // lse / delta of the chunk's 32 queries while the TMEM loads are in flight
+    float4 ls[8], de[8];
+    const float4* lse4 = reinterpret_cast<const float4*>(lse2 + c0);
+    const float4* del4 = reinterpret_cast<const float4*>(delta + c0);
+#pragma unroll
+    for (int t = 0; t < 8; ++t) { ls[t] = lse4[t]; de[t] = del4[t]; }
+    tmem_ld_wait();
+    uint32_t p_pack[16], ds_pack[16];
+#pragma unroll
+    for (int t = 0; t < 32; t += 4) {
+        float p0 = ex2(fmaf(__uint_as_float(s_buf[t]), sl2, -ls[t / 4].x));
+        float p1 = ex2(fmaf(__uint_as_float(s_buf[t + 1]), sl2, -ls[t / 4].y));
+        float p2 = ex2(fmaf(__uint_as_float(s_buf[t + 2]), sl2, -ls[t / 4].z));
+        float p3 = ex2(fmaf(__uint_as_float(s_buf[t + 3]), sl2, -ls[t / 4].w));
+        if (MASKED) {
+            p0 = (c0 + t >= c_lo && c0 + t < c_hi) ? p0 : 0.f;
+            p1 = (c0 + t + 1 >= c_lo && c0 + t + 1 < c_hi) ? p1 : 0.f;
+            p2 = (c0 + t + 2 >= c_lo && c0 + t + 2 < c_hi) ? p2 : 0.f;
+            p3 = (c0 + t + 3 >= c_lo && c0 + t + 3 < c_hi) ? p3 : 0.f;
+        }
+        const float d0 = p0 * (__uint_as_float(dp_buf[t]) - de[t / 4].x);
+        const float d1 = p1 * (__uint_as_float(dp_buf[t + 1]) - de[t / 4].y);
+        const float d2 = p2 * (__uint_as_float(dp_buf[t + 2]) - de[t / 4].z);
+        const float d3 = p3 * (__uint_as_float(dp_buf[t + 3]) - de[t / 4].w);
+        p_pack[t / 2] = pack_bf16(p0, p1);
+        p_pack[t / 2 + 1] = pack_bf16(p2, p3);
+        ds_pack[t / 2] = pack_bf16(d0, d1);
+        ds_pack[t / 2 + 1] = pack_bf16(d2, d3);
+    }
+    tmem_st16(lane_base + COL_ST + cbase + c * 16, p_pack);
+    tmem_st16(lane_base + COL_DPT + cbase + c * 16, ds_pack);
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch) {
+        const int piece = c * 4 + ch;
+        const uint4 val = make_uint4(ds_pack[4 * ch], ds_pack[4 * ch + 1], ds_pack[4 * ch + 2], ds_pack[4 * ch + 3]);
+        *reinterpret_cast<uint4*>(ds_row + ((piece ^ (j & 7)) << 4)) = val;
+    }
+}
+
 // Work items of one block.  Item g is tile g % n_work of head g / n_work; items are ordered head by
 // head (a head's Q and dO tiles stay in L2 while its key tiles are processed) and every block takes a
 // contiguous run of items of about the same total cost (steps plus a constant per item).
@@ -470,7 +521,7 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
         const float sl2 = args.scale_log2;
         const int ds_row_off = (j >> 3) * 1024 + (j & 7) * 128;
-        uint32_t s_buf[32], dp_buf[32];
+        uint32_t s_buf[32], dp_buf[32];                     // K / V row on its way to TMEM; dK / dV row at the end of an item
         bool ok = true;
         int gs = 0;                                         // steps seen so far (aux ring, dS buffer parity)
         int nsh = 0;                                        // non-empty halves of this warpgroup seen so far
@@ -517,52 +568,14 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     ++nsh;
                     tc_fence_after();
                     uint8_t* ds_row = sm.ds[gs & 1][h] + ds_row_off;
+                    // 32 query columns at a time; tiles whose rows all see every column skip the mask code
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {           // 32 query columns at a time
+                    for (int c = 0; c < 2; ++c) {
                         if (c * 32 < n_cols) {
-                            const int c0 = cbase + c * 32;  // first query column of the chunk inside the step
-                            tmem_ld32(lane_base + COL_ST + c0, s_buf);
-                            tmem_ld32(lane_base + COL_DPT + c0, dp_buf);
-                            // lse / delta of the chunk's 32 queries while the TMEM loads are in flight
-                            float4 ls[8], de[8];
-                            const float4* lse4 = reinterpret_cast<const float4*>(&sm.lse2[aslot][c0]);
-                            const float4* del4 = reinterpret_cast<const float4*>(&sm.delta[aslot][c0]);
-#pragma unroll
-                            for (int t = 0; t < 8; ++t) { ls[t] = lse4[t]; de[t] = del4[t]; }
-                            tmem_ld_wait();
-                            uint32_t p_pack[16], ds_pack[16];
-#pragma unroll
-                            for (int t = 0; t < 32; t += 4) {
-                                float p0 = ex2(fmaf(__uint_as_float(s_buf[t]), sl2, -ls[t / 4].x));
-                                float p1 = ex2(fmaf(__uint_as_float(s_buf[t + 1]), sl2, -ls[t / 4].y));
-                                float p2 = ex2(fmaf(__uint_as_float(s_buf[t + 2]), sl2, -ls[t / 4].z));
-                                float p3 = ex2(fmaf(__uint_as_float(s_buf[t + 3]), sl2, -ls[t / 4].w));
-                                if (tile_masked) {
-                                    p0 = (c0 + t >= c_lo && c0 + t < c_hi) ? p0 : 0.f;
-                                    p1 = (c0 + t + 1 >= c_lo && c0 + t + 1 < c_hi) ? p1 : 0.f;
-                                    p2 = (c0 + t + 2 >= c_lo && c0 + t + 2 < c_hi) ? p2 : 0.f;
-                                    p3 = (c0 + t + 3 >= c_lo && c0 + t + 3 < c_hi) ? p3 : 0.f;
-                                }
-                                const float d0 = p0 * (__uint_as_float(dp_buf[t]) - de[t / 4].x);
-                                const float d1 = p1 * (__uint_as_float(dp_buf[t + 1]) - de[t / 4].y);
-                                const float d2 = p2 * (__uint_as_float(dp_buf[t + 2]) - de[t / 4].z);
-                                const float d3 = p3 * (__uint_as_float(dp_buf[t + 3]) - de[t / 4].w);
-                                p_pack[t / 2] = pack_bf16(p0, p1);
-                                p_pack[t / 2 + 1] = pack_bf16(p2, p3);
-                                ds_pack[t / 2] = pack_bf16(d0, d1);
-                                ds_pack[t / 2 + 1] = pack_bf16(d2, d3);
-                            }
-                            // P^T over S^T and dS^T over dP^T: the 16 packed columns of chunk c start at column
-                            // c * 16 of the half, which this thread has already read
-                            tmem_st16(lane_base + COL_ST + cbase + c * 16, p_pack);
-                            tmem_st16(lane_base + COL_DPT + cbase + c * 16, ds_pack);
-                            // dS^T to shared memory: 4 pieces of 8 queries, 128-byte swizzle on the key row
-#pragma unroll
-                            for (int ch = 0; ch < 4; ++ch) {
-                                const int piece = c * 4 + ch;
-                                uint4 val = make_uint4(ds_pack[4 * ch], ds_pack[4 * ch + 1], ds_pack[4 * ch + 2], ds_pack[4 * ch + 3]);
-                                *reinterpret_cast<uint4*>(ds_row + ((piece ^ (j & 7)) << 4)) = val;
-                            }
+                            if (tile_masked)
+                                softmax_grad_chunk<true>(lane_base, cbase, c, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi, ds_row, j);
+                            else
+                                softmax_grad_chunk<false>(lane_base, cbase, c, sm.lse2[aslot], sm.delta[aslot], sl2, 0, 0, ds_row, j);
                         }
                     }
                     tmem_st_wait();

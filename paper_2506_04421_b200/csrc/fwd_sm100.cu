@@ -44,7 +44,7 @@ struct __align__(1024) SharedStorage {
     uint8_t v[NSTAGE][TILE_BYTES];
     uint64_t q_full, q_tmem;
     uint64_t k_full[NSTAGE], k_empty[NSTAGE], v_full[NSTAGE], v_empty[NSTAGE];
-    uint64_t s_full[2], p_full[2], pv_done;
+    uint64_t s_full[2], p_full[2], pv_done, o_done;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -128,6 +128,7 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             mbar_init(&sm.p_full[h], 128);
         }
         mbar_init(&sm.pv_done, 1);
+        mbar_init(&sm.o_done, 1);
         fence_mbar_init();
     }
     if (warp == 1) {
@@ -235,11 +236,18 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 for (int ks = 0; ks < HN / 16; ++ks)
                     if (ks < nk)
                         mma_ts(tmem + COL_O, tmem + COL_S + h * HN + ks * 8, vd + ks * 128, idesc_pv, !first || (ks > 0));
-                tc_commit(&sm.pv_done);
-                if (h == 1 || half_cols(n_valid, 1) == 0) {      // last half of the tile
+                // Nobody waits for the slots of the last NSTAGE tiles to become free, and the block may exit as
+                // soon as the softmax warps have seen the last pv_done: an arrival that lands after that would
+                // hit the barriers of the next block on this SM.  So those slots are not signalled at all, and
+                // pv_done / o_done are signalled last.
+                if ((h == 1 || half_cols(n_valid, 1) == 0) && j + NSTAGE < n_tiles) {      // last half of the tile
                     tc_commit(&sm.k_empty[slot]);
                     tc_commit(&sm.v_empty[slot]);
                 }
+                tc_commit(&sm.pv_done);
+                // the last product of the block also completes o_done, which the epilogue waits for: a warp
+                // may be two halves ahead of the tensor core there, too far for pv_done's parity to tell
+                if (j + 1 == n_tiles && (h == 1 || half_cols(n_valid, 1) == 0)) tc_commit(&sm.o_done);
             }
             __syncwarp();
             return true;
@@ -386,7 +394,7 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
 
         if (ok) {
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.pv_done, (pv_issued - 1) & 1, abort_flag));
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_done, 0, abort_flag));
             if (!ok && lane == 0) report_timeout(args.status, 0xA00);
         }
         if (ok) {

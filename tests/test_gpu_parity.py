@@ -191,6 +191,27 @@ def test_scale_step_full_batch_last_scales_sampled_heads():
     _no_device_error()
 
 
+def test_full_size_forward_and_scale_step_repeat_bit_identical():
+    """The forward paths have no atomics, so two runs on the same inputs must agree bit for bit, at the
+    sizes where thousands of blocks start and finish at different times (a warp that reads its output
+    accumulator before the last product has landed shows up here)."""
+    wl = CONFIGS["512_d24_infer"]
+    s = len(wl.side_lens) - 1
+    side, side_prev = wl.side_lens[s], wl.side_lens[s - 1]
+    t = [bulk_normal(wl.seed, i, wl.B, wl.H, (side_prev if i in (1, 2) else side) ** 2, wl.D) for i in range(5)]
+    first, _ = hmar.hmar_attn_scale_step(*t, side_prev, side, wl.softmax_scale)
+    for _ in range(4):
+        again, _ = hmar.hmar_attn_scale_step(*t, side_prev, side, wl.softmax_scale)
+        assert torch.equal(first, again)
+    wt = CONFIGS["512_d24_train"]
+    q, k, v = (bulk_normal(wt.seed, i, wt.B, wt.H, wt.L, wt.D) for i in range(3))
+    o1, l1 = hmar.hmar_attn_fwd(q, k, v, wt.side_lens, wt.softmax_scale)
+    for _ in range(3):
+        o2, l2 = hmar.hmar_attn_fwd(q, k, v, wt.side_lens, wt.softmax_scale)
+        assert torch.equal(o1, o2) and torch.equal(l1, l2)
+    _no_device_error()
+
+
 def test_scale_step_matches_training_forward_rows():
     """The inference step of scale k equals the scale-k rows of the training forward (same kernels'
     arithmetic, different entry point)."""
