@@ -3,16 +3,23 @@
 // One block handles one work tile: up to 128 consecutive query rows of one head and the contiguous
 // key range those rows may see under the mask (paper Sec. 4.1, Fig. attn-mask).  It is the usual
 // IO-aware tiling with an online softmax (Sec. 4.1: the kernel extends FlashAttention), laid out for
-// Blackwell:
-//   warp 0      TMA producer: Q once, then K and V tiles of 128 keys through a shared-memory ring
-//   warp 1      issues tcgen05.mma.  Q is copied to TMEM once and is the A operand of S = Q K^T; a key
-//               tile is handled as two halves of 64 keys with their own S columns and barriers, so the
-//               tensor core computes one half while the softmax warps work on the other.  P replaces S
-//               in place (bf16) and is the TMEM A operand of O += P V.
-//   warps 2-5   one query row per thread.  A half's 64 logits are read from TMEM once; the running
-//               maximum is kept unless the half exceeds it by more than 2^8 (then O and the row sum are
-//               rescaled first), P = 2^(s - m) goes back to TMEM as bf16.
-// TMEM columns: S/P half a [0,64), half b [64,128), O [128,192), Q [192,224).  Two blocks fit on one SM.
+// Blackwell.  Every 128-key tile is split into two halves of 64 keys, and each half has its own softmax
+// warpgroup, its own running maximum and row sum, and its own output accumulator: the two halves are
+// two independent attention problems over disjoint key sets, merged exactly at the end
+// (O = (w_a O_a + w_b O_b) / (w_a l_a + w_b l_b), w_x = 2^(m_x - max(m_a, m_b))).  Nothing ties the two
+// chains together, so one waits for the tensor core while the other computes, and two blocks per SM
+// give four such chains.
+//   warps 0-3   softmax of half a: one query row per thread, 64 logits per tile read from TMEM once; the
+//               running maximum is kept unless the tile exceeds it by more than 2^8 (then O_a and the
+//               row sum are rescaled first), P = 2^(s - m) goes back to TMEM as bf16 over S
+//   warps 4-7   the same for half b
+//   warp 8      TMA producer: Q once, then K and V tiles of 128 keys through a shared-memory ring
+//   warp 9      issues tcgen05.mma: S_x = Q K_x^T (both operands in shared memory), O_x += P_x V_x (P_x from
+//               TMEM, V_x an MN-major shared-memory operand), one burst per half and tile:
+//               O_x += P_x V_x of tile j, then S_x of tile j + 1 into the columns P_x has just left
+// TMEM columns: S/P of half a [0,64), of half b [64,128), O_a [128,192), O_b [192,256).
+// Registers: the block starts with 80 per thread (two blocks per SM); the softmax warpgroups raise
+// theirs to 96 and the third warpgroup drops to 48 (setmaxnreg), the same total.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -33,18 +40,23 @@ constexpr int HN = 64;               // keys per half tile
 constexpr int D = kHeadDim;
 constexpr int NSTAGE = 2;
 constexpr int TILE_BYTES = BN * D * 2;          // 16 KB
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 384;
+constexpr int NUM_SOFTMAX_THREADS = 256;
+constexpr int PRODUCER_WARP = 8, MMA_WARP = 9;
+constexpr int REGS_START = 80, REGS_SOFTMAX = 96, REGS_MISC = 48;
+static_assert(2 * REGS_SOFTMAX + REGS_MISC == 3 * REGS_START, "register budget of the block");
 constexpr uint32_t TMEM_COLS = 256;
-constexpr uint32_t COL_S = 0, COL_O = 128, COL_Q = 192;
+constexpr uint32_t COL_S = 0, COL_O = 128;
 constexpr float kRescaleThreshold = 8.0f;       // in log2 units
 
 struct __align__(1024) SharedStorage {
     uint8_t q[TILE_BYTES];
     uint8_t k[NSTAGE][TILE_BYTES];
     uint8_t v[NSTAGE][TILE_BYTES];
-    uint64_t q_full, q_tmem;
+    float2 stats[2][BM];                     // (running maximum, row sum) of each half, for the merge
+    uint64_t q_full;
     uint64_t k_full[NSTAGE], k_empty[NSTAGE], v_full[NSTAGE], v_empty[NSTAGE];
-    uint64_t s_full[2], p_full[2], pv_done, o_done;
+    uint64_t s_full[2], p_full[2], o_done, stats_ready;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -82,6 +94,13 @@ __device__ __forceinline__ void report_timeout(int* status, int where) {
     }
 }
 
+template <int N> __device__ __forceinline__ void reg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N> __device__ __forceinline__ void reg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 2)
 hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k0,
                    const __grid_constant__ CUtensorMap map_v0, const __grid_constant__ CUtensorMap map_k1,
@@ -116,7 +135,6 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     if (threadIdx.x == 0) {
         sm.abort_flag = 0;
         mbar_init(&sm.q_full, 1);
-        mbar_init(&sm.q_tmem, 128);
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(&sm.k_full[s], 1);
             mbar_init(&sm.k_empty[s], 1);
@@ -125,13 +143,13 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
         for (int h = 0; h < 2; ++h) {
             mbar_init(&sm.s_full[h], 1);
-            mbar_init(&sm.p_full[h], 128);
+            mbar_init(&sm.p_full[h], NUM_SOFTMAX_THREADS / 2);
         }
-        mbar_init(&sm.pv_done, 1);
         mbar_init(&sm.o_done, 1);
+        mbar_init(&sm.stats_ready, NUM_SOFTMAX_THREADS);
         fence_mbar_init();
     }
-    if (warp == 1) {
+    if (warp == MMA_WARP) {
         tmem_alloc(&sm.tmem_base, TMEM_COLS);
         tmem_relinquish();
     }
@@ -141,129 +159,137 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     const uint32_t tmem = sm.tmem_base;
     volatile int* abort_flag = &sm.abort_flag;
 
-    if (warp == 0) {
-        // ================================================================== TMA producer
-        // The whole warp runs the control flow; one elected lane issues the copies (a warp that has split
-        // into one running lane and 31 parked ones issues far more slowly).
-        const bool leader = elect_one();
-        if (leader) {
-            prefetch_tensormap(&map_q);
-            prefetch_tensormap(&map_k0);
-            prefetch_tensormap(&map_v0);
-            mbar_arrive_expect_tx(&sm.q_full, TILE_BYTES);
-            tma_load_3d(sm.q, &map_q, &sm.q_full, 0, w.row_begin, bh);
-        }
-        __syncwarp();
-        bool ok = true;
-        for (int j = 0; j < n_tiles && ok; ++j) {
-            const int slot = j % NSTAGE;
-            const uint32_t par = ((j / NSTAGE) & 1) ^ 1;     // parity of the previous use of the slot
-            const KvTile t = kv_tile(w, tiles0, j);
-            if (j >= NSTAGE) ok = __all_sync(0xffffffffu, mbar_wait(&sm.k_empty[slot], par, abort_flag));
-            if (!ok) { if (lane == 0) report_timeout(args.status, 0x100 + j); break; }
+    if (warp >= PRODUCER_WARP) {
+        reg_dec<REGS_MISC>();
+        if (warp == PRODUCER_WARP) {
+            // ================================================================== TMA producer
+            // The whole warp runs the control flow; one elected lane issues the copies (a warp that has split
+            // into one running lane and 31 parked ones issues far more slowly).
+            const bool leader = elect_one();
             if (leader) {
-                mbar_arrive_expect_tx(&sm.k_full[slot], TILE_BYTES);
-                tma_load_3d(sm.k[slot], t.seg ? &map_k1 : &map_k0, &sm.k_full[slot], 0, t.coord, bh);
+                prefetch_tensormap(&map_q);
+                prefetch_tensormap(&map_k0);
+                prefetch_tensormap(&map_v0);
+                mbar_arrive_expect_tx(&sm.q_full, TILE_BYTES);
+                tma_load_3d(sm.q, &map_q, &sm.q_full, 0, w.row_begin, bh);
             }
             __syncwarp();
-            if (j >= NSTAGE) ok = __all_sync(0xffffffffu, mbar_wait(&sm.v_empty[slot], par, abort_flag));
-            if (!ok) { if (lane == 0) report_timeout(args.status, 0x200 + j); break; }
-            if (leader) {
-                mbar_arrive_expect_tx(&sm.v_full[slot], TILE_BYTES);
-                tma_load_3d(sm.v[slot], t.seg ? &map_v1 : &map_v0, &sm.v_full[slot], 0, t.coord, bh);
+            bool ok = true;
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int slot = j % NSTAGE;
+                const uint32_t par = ((j / NSTAGE) & 1) ^ 1;     // parity of the previous use of the slot
+                const KvTile t = kv_tile(w, tiles0, j);
+                if (j >= NSTAGE) ok = __all_sync(0xffffffffu, mbar_wait(&sm.k_empty[slot], par, abort_flag));
+                if (!ok) { if (lane == 0) report_timeout(args.status, 0x100 + j); break; }
+                if (leader) {
+                    mbar_arrive_expect_tx(&sm.k_full[slot], TILE_BYTES);
+                    tma_load_3d(sm.k[slot], t.seg ? &map_k1 : &map_k0, &sm.k_full[slot], 0, t.coord, bh);
+                }
+                __syncwarp();
+                if (j >= NSTAGE) ok = __all_sync(0xffffffffu, mbar_wait(&sm.v_empty[slot], par, abort_flag));
+                if (!ok) { if (lane == 0) report_timeout(args.status, 0x200 + j); break; }
+                if (leader) {
+                    mbar_arrive_expect_tx(&sm.v_full[slot], TILE_BYTES);
+                    tma_load_3d(sm.v[slot], t.seg ? &map_v1 : &map_v0, &sm.v_full[slot], 0, t.coord, bh);
+                }
+                __syncwarp();
             }
-            __syncwarp();
-        }
-        if (!ok) {
-            // give the copies already issued a bounded chance to land before the block exits
-            const uint64_t t0 = globaltimer_ns();
-            while (globaltimer_ns() - t0 < 2000000ull) { }
-        }
-    } else if (warp == 1) {
-        // ================================================================== MMA issuer
-        // The whole warp runs the control flow; one elected lane issues.  Descriptors are built once and
-        // advanced by adding (byte offset >> 4), so issuing an MMA costs a few instructions.
-        const bool leader = elect_one();
-        const uint64_t k_kd0 = smem_desc_sw128(smem_u32(sm.k[0]), 16);      // ring slots are 16 KB apart
-        const uint64_t v_mn0 = smem_desc_sw128(smem_u32(sm.v[0]), 1024);
-        constexpr uint32_t idesc_pv = idesc_bf16_f32(BM, D, false, true);
-        int p_seen[2] = {0, 0};                                 // completed phases of p_full[h] consumed so far
-        bool ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_tmem, 0, abort_flag));
-        if (!ok && lane == 0) report_timeout(args.status, 0x300);
-
-        // S_h = Q K_h^T for half h of tile j (Q from TMEM, 64 keys of the tile from shared memory)
-        auto issue_s = [&](int j, int h) -> bool {
-            const int slot = j % NSTAGE;
-            const int n = half_cols(kv_tile(w, tiles0, j).n_valid, h);
-            if (n == 0) return true;
-            if (h == 0 && !__all_sync(0xffffffffu, mbar_wait(&sm.k_full[slot], (j / NSTAGE) & 1, abort_flag))) {
-                if (lane == 0) report_timeout(args.status, 0x400 + j);
+            if (!ok) {
+                // give the copies already issued a bounded chance to land before the block exits
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 2000000ull) { }
+            }
+        } else if (warp == MMA_WARP) {
+            // ================================================================== MMA issuer
+            // The whole warp runs the control flow; one elected lane issues.  Descriptors are built once and
+            // advanced by adding (byte offset >> 4), so issuing an MMA costs a few instructions.
+            const bool leader = elect_one();
+            const uint64_t q_kd = smem_desc_sw128(smem_u32(sm.q), 16);
+            const uint64_t k_kd0 = smem_desc_sw128(smem_u32(sm.k[0]), 16);      // ring slots are 16 KB apart
+            const uint64_t v_mn0 = smem_desc_sw128(smem_u32(sm.v[0]), 1024);
+            constexpr uint32_t idesc_pv = idesc_bf16_f32(BM, D, false, true);
+            uint32_t par_p[2] = {0, 0};                             // parity of the next p_full[h] phase
+            bool o_started[2] = {false, false};                     // O_x has received a product
+            auto wait = [&](uint64_t* bar, uint32_t parity, int code) -> bool {
+                if (__all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag))) return true;
+                if (lane == 0) report_timeout(args.status, code);
                 return false;
-            }
-            tc_fence_after();
-            if (leader) {
+            };
+            // S_h = Q K_h^T for n keys of half h of the tile in ring slot `slot`
+            auto issue_s = [&](int h, int n, int slot) {
                 const uint32_t idesc = idesc_bf16_f32(BM, n, false, false);
                 const uint64_t kd = k_kd0 + slot * 1024 + h * 512;              // + 64 rows
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ts(tmem + COL_S + h * HN, tmem + COL_Q + ks * 8, kd + ks * 2, idesc, ks > 0);
+                    mma_ss(tmem + COL_S + h * HN, q_kd + ks * 2, kd + ks * 2, idesc, ks > 0);
                 tc_commit(&sm.s_full[h]);
-            }
-            __syncwarp();
-            return true;
-        };
-        // O += P_h V_h for half h of tile j; the tile's last half releases its K and V slots
-        auto issue_pv = [&](int j, int h) -> bool {
-            const int slot = j % NSTAGE;
-            const int n_valid = kv_tile(w, tiles0, j).n_valid;
-            const int n = half_cols(n_valid, h);
-            if (n == 0) return true;
-            const int par = h == 0 ? (p_seen[0]++ & 1) : (p_seen[1]++ & 1);
-            if (!__all_sync(0xffffffffu, mbar_wait(&sm.p_full[h], par, abort_flag))) {
-                if (lane == 0) report_timeout(args.status, 0x600 + j);
-                return false;
-            }
-            if (h == 0 && !__all_sync(0xffffffffu, mbar_wait(&sm.v_full[slot], (j / NSTAGE) & 1, abort_flag))) {
-                if (lane == 0) report_timeout(args.status, 0x500 + j);
-                return false;
-            }
-            tc_fence_after();
-            if (leader) {
+            };
+            // O_h += P_h V_h for n keys of half h
+            auto issue_pv = [&](int h, int n, int slot) {
                 const int nk = n / 16;
                 const uint64_t vd = v_mn0 + slot * 1024 + h * 512;
-                const bool first = (j == 0) && (h == 0);
 #pragma unroll
                 for (int ks = 0; ks < HN / 16; ++ks)
                     if (ks < nk)
-                        mma_ts(tmem + COL_O, tmem + COL_S + h * HN + ks * 8, vd + ks * 128, idesc_pv, !first || (ks > 0));
-                // Nobody waits for the slots of the last NSTAGE tiles to become free, and the block may exit as
-                // soon as the softmax warps have seen the last pv_done: an arrival that lands after that would
-                // hit the barriers of the next block on this SM.  So those slots are not signalled at all, and
-                // pv_done / o_done are signalled last.
-                if ((h == 1 || half_cols(n_valid, 1) == 0) && j + NSTAGE < n_tiles) {      // last half of the tile
-                    tc_commit(&sm.k_empty[slot]);
-                    tc_commit(&sm.v_empty[slot]);
-                }
-                tc_commit(&sm.pv_done);
-                // the last product of the block also completes o_done, which the epilogue waits for: a warp
-                // may be two halves ahead of the tensor core there, too far for pv_done's parity to tell
-                if (j + 1 == n_tiles && (h == 1 || half_cols(n_valid, 1) == 0)) tc_commit(&sm.o_done);
-            }
-            __syncwarp();
-            return true;
-        };
+                        mma_ts(tmem + COL_O + h * HN, tmem + COL_S + h * HN + ks * 8, vd + ks * 128, idesc_pv,
+                               o_started[h] || (ks > 0));
+                o_started[h] = true;
+            };
 
-        if (ok) ok = issue_s(0, 0);
-        if (ok) ok = issue_s(0, 1);
-        for (int j = 0; j < n_tiles && ok; ++j) {
-            ok = issue_pv(j, 0);
-            if (ok && j + 1 < n_tiles) ok = issue_s(j + 1, 0);
-            if (ok) ok = issue_pv(j, 1);
-            if (ok && j + 1 < n_tiles) ok = issue_s(j + 1, 1);
+            bool ok = wait(&sm.q_full, 0, 0x300) && wait(&sm.k_full[0], 0, 0x400);
+            if (ok) {
+                tc_fence_after();
+                const int nv = kv_tile(w, tiles0, 0).n_valid;
+                if (leader) {
+                    issue_s(0, half_cols(nv, 0), 0);
+                    if (half_cols(nv, 1) > 0) issue_s(1, half_cols(nv, 1), 0);
+                    if (NSTAGE < n_tiles) tc_commit(&sm.k_empty[0]);
+                }
+                __syncwarp();
+            }
+            for (int j = 0; j < n_tiles && ok; ++j) {
+                const int slot = j % NSTAGE, slot_next = (j + 1) % NSTAGE;
+                const bool more = j + 1 < n_tiles;
+                const int nv = kv_tile(w, tiles0, j).n_valid;
+                const int nv_next = more ? kv_tile(w, tiles0, j + 1).n_valid : 0;
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int n = half_cols(nv, h), n_next = half_cols(nv_next, h);
+                    // one burst: O_h += P_h V_h of tile j, then S_h of tile j + 1 over the columns P_h leaves
+                    if (n > 0) {
+                        ok = wait(&sm.p_full[h], par_p[h], 0x600 + j);
+                        par_p[h] ^= 1;
+                    }
+                    if (ok && h == 0) {
+                        ok = wait(&sm.v_full[slot], (j / NSTAGE) & 1, 0x500 + j);
+                        if (ok && more) ok = wait(&sm.k_full[slot_next], ((j + 1) / NSTAGE) & 1, 0x400 + j);
+                    }
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (leader) {
+                        if (n > 0) issue_pv(h, n, slot);
+                        if (n_next > 0) issue_s(h, n_next, slot_next);
+                        if (h == 1) {
+                            // V of tile j and K of tile j + 1 have been handed to their last readers; a slot is
+                            // signalled free only if a later tile will use it (the block may exit as soon as the
+                            // softmax warps have seen o_done: an arrival that lands after that would hit the
+                            // barriers of the next block on this SM)
+                            if (j + NSTAGE < n_tiles) tc_commit(&sm.v_empty[slot]);
+                            if (j + 1 + NSTAGE < n_tiles) tc_commit(&sm.k_empty[slot_next]);
+                            if (!more) tc_commit(&sm.o_done);
+                        }
+                    } else if (n > 0) {
+                        o_started[h] = true;
+                    }
+                    __syncwarp();
+                }
+            }
         }
     } else {
-        // ================================================================== softmax + epilogue
+        // ================================================================== softmax warpgroups + epilogue
+        reg_inc<REGS_SOFTMAX>();
         const int quarter = warp & 3;
+        const int h = warp >> 2;                               // the half of every tile this warpgroup owns
         const int r = quarter * 32 + lane;                     // row inside the tile
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
         const int row = w.row_begin + r;
@@ -275,158 +301,156 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             hi = args.st.start[s + 1];
         }
         const float sl2 = args.scale_log2;
+        const int col0 = h * HN;                               // first key of this half inside a tile
+        const uint32_t s_addr = lane_base + COL_S + col0;
+        const uint32_t o_addr = lane_base + COL_O + col0;
         float m_used = -INFINITY, l = 0.f;
         bool ok = true;
-        int pv_issued = 0;                                     // halves handed to the tensor core so far
-        int s_seen[2] = {0, 0};                                // completed phases of s_full[h] consumed so far
+        bool have_o = false;                                   // O_h has received a product
+        uint32_t par_s = 0;                                    // parity of the next s_full[h] phase
         uint32_t b0[32], b1[32];
-
-        // ---- Q row to TMEM (A operand of S = Q K^T): undo the 128-byte swizzle of the TMA tile
-        ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_full, 0, abort_flag));
-        if (!ok && lane == 0) report_timeout(args.status, 0x700);
-        if (ok) {
-            const uint8_t* qrow = sm.q + r * 128;
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                const uint4 val = *reinterpret_cast<const uint4*>(qrow + ((c ^ (r & 7)) << 4));
-                b0[4 * c] = val.x; b0[4 * c + 1] = val.y; b0[4 * c + 2] = val.z; b0[4 * c + 3] = val.w;
-            }
-            tmem_st32(lane_base + COL_Q, b0);
-            tmem_st_wait();
-            tc_fence_before();
-            mbar_arrive(&sm.q_tmem);
-        }
 
         for (int j = 0; j < n_tiles && ok; ++j) {
             const KvTile t = kv_tile(w, tiles0, j);
+            const int n = half_cols(t.n_valid, h);
+            if (n == 0) continue;
             // key c of the tile is visible to this row iff c in [c_lo, c_hi)
             const int c_lo = w.uniform ? 0 : max(lo - t.coord, 0);
             const int c_hi = w.uniform ? t.n_valid : min(hi - t.coord, t.n_valid);
+            const bool two = n > 32;                           // second 32-column chunk present
+            const bool need_mask = (!w.uniform) || (t.n_valid < col0 + (two ? 64 : 32));
 
-            for (int h = 0; h < 2 && ok; ++h) {
-                const int n = half_cols(t.n_valid, h);
-                if (n == 0) break;
-                const int col0 = h * HN;                           // first key of the half inside the tile
-                const bool two = n > 32;                           // second 32-column chunk present
-                const bool need_mask = (!w.uniform) || (t.n_valid < col0 + (two ? 64 : 32));
-                const uint32_t s_addr = lane_base + COL_S + col0;
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[h], par_s, abort_flag));
+            if (!ok) { if (lane == 0) report_timeout(args.status, 0x800 + j); break; }
+            par_s ^= 1;
+            tc_fence_after();
 
-                const int par = h == 0 ? (s_seen[0]++ & 1) : (s_seen[1]++ & 1);
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[h], par, abort_flag));
-                if (!ok) { if (lane == 0) report_timeout(args.status, 0x800 + j); break; }
-                tc_fence_after();
+            tmem_ld32(s_addr, b0);
+            if (two) tmem_ld32(s_addr + 32, b1);
+            tmem_ld_wait();
 
-                tmem_ld32(s_addr, b0);
-                if (two) tmem_ld32(s_addr + 32, b1);
-                tmem_ld_wait();
-
-                // masked logits become -inf once, so the maximum and the exponentials treat them alike
-                if (need_mask) {
+            // masked logits become -inf once, so the maximum and the exponentials treat them alike
+            if (need_mask) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        if (!(col0 + i >= c_lo && col0 + i < c_hi)) b0[i] = 0xff800000u;
-                        if (!(col0 + 32 + i >= c_lo && col0 + 32 + i < c_hi)) b1[i] = 0xff800000u;
+                for (int i = 0; i < 32; ++i) {
+                    if (!(col0 + i >= c_lo && col0 + i < c_hi)) b0[i] = 0xff800000u;
+                    if (!(col0 + 32 + i >= c_lo && col0 + 32 + i < c_hi)) b1[i] = 0xff800000u;
+                }
+            }
+            float mx = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(b0[i]));
+            if (two) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(b1[i]));
+            }
+            mx *= sl2;                                          // softmax_scale > 0
+
+            // Keep the running maximum unless this tile exceeds it by more than the threshold.  O_h is
+            // quiet here: the product that precedes S_h of this tile in the tensor core's queue is the
+            // last one that wrote it, and the next one waits for this warpgroup.
+            const bool grow = mx > m_used + kRescaleThreshold;  // false for -inf > -inf
+            if (__any_sync(0xffffffffu, grow)) {
+                const float m_new = fmaxf(m_used, mx);
+                const float f = (m_used == -INFINITY) ? 0.f : ex2(m_used - m_new);
+                m_used = m_new;
+                l *= f;
+                if (have_o) {
+#pragma unroll 1
+                    for (int piece = 0; piece < 4; ++piece) {
+                        uint32_t o[16];
+                        tmem_ld16(o_addr + piece * 16, o);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
+                        tmem_st16(o_addr + piece * 16, o);
                     }
                 }
-                float mx = -INFINITY;
-#pragma unroll
-                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(b0[i]));
-                if (two) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(b1[i]));
-                }
-                mx *= sl2;                                          // softmax_scale > 0
+            }
+            const float m_sub = (m_used == -INFINITY) ? 0.f : m_used;
 
-                // Keep the running maximum unless this half exceeds it by more than the threshold.
-                const bool grow = mx > m_used + kRescaleThreshold;  // false for -inf > -inf
-                if (__any_sync(0xffffffffu, grow)) {
-                    // O must be quiet: wait for every P V product handed over so far
-                    if (pv_issued > 0) {
-                        ok = __all_sync(0xffffffffu, mbar_wait(&sm.pv_done, (pv_issued - 1) & 1, abort_flag));
-                        if (!ok) { if (lane == 0) report_timeout(args.status, 0x900 + j); break; }
-                        tc_fence_after();
-                    }
-                    const float m_new = fmaxf(m_used, mx);
-                    const float f = (m_used == -INFINITY) ? 0.f : ex2(m_used - m_new);
-                    m_used = m_new;
-                    l *= f;
-                    if (pv_issued > 0) {
-                        uint32_t o[32];
+            // P = 2^(s * scale - m): fp32 row sum, bf16 P written over the S columns already read
+            uint32_t packed[16];
+            float l_add = 0.f;
 #pragma unroll
-                        for (int hh = 0; hh < 2; ++hh) {
-                            tmem_ld32(lane_base + COL_O + hh * 32, o);
-                            tmem_ld_wait();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) o[i] = __float_as_uint(__uint_as_float(o[i]) * f);
-                            tmem_st32(lane_base + COL_O + hh * 32, o);
-                        }
-                    }
-                }
-                const float m_sub = (m_used == -INFINITY) ? 0.f : m_used;
-
-                // P = 2^(s * scale - m): fp32 row sum, bf16 P written over the S columns already read
-                uint32_t packed[16];
-                float l_add = 0.f;
+            for (int i = 0; i < 32; i += 2) {
+                const float p0 = ex2(fmaf(__uint_as_float(b0[i]), sl2, -m_sub));
+                const float p1 = ex2(fmaf(__uint_as_float(b0[i + 1]), sl2, -m_sub));
+                l_add += p0 + p1;
+                packed[i / 2] = pack_bf16(p0, p1);
+            }
+            tmem_st16(s_addr, packed);
+            if (two) {
 #pragma unroll
                 for (int i = 0; i < 32; i += 2) {
-                    const float p0 = ex2(fmaf(__uint_as_float(b0[i]), sl2, -m_sub));
-                    const float p1 = ex2(fmaf(__uint_as_float(b0[i + 1]), sl2, -m_sub));
+                    const float p0 = ex2(fmaf(__uint_as_float(b1[i]), sl2, -m_sub));
+                    const float p1 = ex2(fmaf(__uint_as_float(b1[i + 1]), sl2, -m_sub));
                     l_add += p0 + p1;
                     packed[i / 2] = pack_bf16(p0, p1);
                 }
-                tmem_st16(s_addr, packed);
-                if (two) {
-#pragma unroll
-                    for (int i = 0; i < 32; i += 2) {
-                        const float p0 = ex2(fmaf(__uint_as_float(b1[i]), sl2, -m_sub));
-                        const float p1 = ex2(fmaf(__uint_as_float(b1[i + 1]), sl2, -m_sub));
-                        l_add += p0 + p1;
-                        packed[i / 2] = pack_bf16(p0, p1);
-                    }
-                    tmem_st16(s_addr + 16, packed);
-                }
-                l += l_add;
-                tmem_st_wait();
-                tc_fence_before();
-                mbar_arrive(&sm.p_full[h]);
-                ++pv_issued;
+                tmem_st16(s_addr + 16, packed);
             }
+            l += l_add;
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(&sm.p_full[h]);
+            have_o = true;
         }
 
+        // ---- merge of the two halves and epilogue: this warpgroup writes output columns [32 h, 32 h + 32)
         if (ok) {
             ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_done, 0, abort_flag));
             if (!ok && lane == 0) report_timeout(args.status, 0xA00);
         }
         if (ok) {
+            sm.stats[h][r] = make_float2(m_used, l);
+            mbar_arrive(&sm.stats_ready);
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.stats_ready, 0, abort_flag));
+            if (!ok && lane == 0) report_timeout(args.status, 0xB00);
+        }
+        if (ok) {
             tc_fence_after();
-            const float inv = 1.f / l;
-            __nv_bfloat16* orow = args.out + ((size_t)bh * args.n_q_rows + row) * D;
+            const float2 sa = sm.stats[0][r], sb = sm.stats[1][r];
+            // half a always has keys; half b has none when every tile of the block is at most 64 keys wide
+            // (its accumulator is then unwritten and must not be read into the result)
+            const bool b_used = sb.y > 0.f;
+            const float m = b_used ? fmaxf(sa.x, sb.x) : sa.x;
+            const float wa = ex2(sa.x - m);
+            const float wb = b_used ? ex2(sb.x - m) : 0.f;
+            const float lsum = sa.y * wa + sb.y * wb;
+            const float inv = 1.f / lsum;
+            const float fa = wa * inv, fb = wb * inv;
+            tmem_ld32(lane_base + COL_O + h * 32, b0);                 // O_a, this warpgroup's 32 columns
+            tmem_ld32(lane_base + COL_O + HN + h * 32, b1);            // O_b
+            tmem_ld_wait();
+            if (row_ok) {
+                __nv_bfloat16* orow = args.out + ((size_t)bh * args.n_q_rows + row) * D + h * 32;
+                uint4* dst = reinterpret_cast<uint4*>(orow);
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                tmem_ld32(lane_base + COL_O + h * 32, b0);
-                tmem_ld_wait();
-                if (row_ok) {
-                    uint4* dst = reinterpret_cast<uint4*>(orow + h * 32);
+                for (int i = 0; i < 4; ++i) {
+                    float o[8];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint4 v4;
-                        v4.x = pack_bf16(__uint_as_float(b0[8 * i + 0]) * inv, __uint_as_float(b0[8 * i + 1]) * inv);
-                        v4.y = pack_bf16(__uint_as_float(b0[8 * i + 2]) * inv, __uint_as_float(b0[8 * i + 3]) * inv);
-                        v4.z = pack_bf16(__uint_as_float(b0[8 * i + 4]) * inv, __uint_as_float(b0[8 * i + 5]) * inv);
-                        v4.w = pack_bf16(__uint_as_float(b0[8 * i + 6]) * inv, __uint_as_float(b0[8 * i + 7]) * inv);
-                        dst[i] = v4;
+                    for (int e = 0; e < 8; ++e) {
+                        const float a = __uint_as_float(b0[8 * i + e]) * fa;
+                        o[e] = b_used ? fmaf(__uint_as_float(b1[8 * i + e]), fb, a) : a;
                     }
+                    uint4 v4;
+                    v4.x = pack_bf16(o[0], o[1]);
+                    v4.y = pack_bf16(o[2], o[3]);
+                    v4.z = pack_bf16(o[4], o[5]);
+                    v4.w = pack_bf16(o[6], o[7]);
+                    dst[i] = v4;
                 }
+                if (h == 0 && args.lse != nullptr)
+                    args.lse[(size_t)bh * args.n_q_rows + row] = (m + log2f(lsum)) * 0.6931471805599453f;
             }
-            if (row_ok && args.lse != nullptr)
-                args.lse[(size_t)bh * args.n_q_rows + row] = (m_used + log2f(l)) * 0.6931471805599453f;
         }
     }
 
     // ---- tear-down
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == MMA_WARP) {
         tc_fence_after();
         tmem_dealloc(tmem, TMEM_COLS);
     }
