@@ -125,6 +125,56 @@ def time_oracle(wl, n_heads, steps, warmup):
                       f"{sec * 1e3:.0f} ms per sample; numpy fp64 with an explicit {wl.L}x{wl.L} mask"}, sec
 
 
+def time_dense_masked(wl, q, k, v, do, reps=3):
+    """Dense masked attention of the same shape on the same GPU (torch SDPA with the explicit boolean HMAR
+    mask, forward + backward): the comparison the paper's App. B.4 makes.  Library kernels, timed outside
+    the benchmark's own timed region; reported as context only."""
+    import torch
+    import torch.nn.functional as F
+    n = [s * s for s in wl.side_lens]
+    scale_of = torch.repeat_interleave(torch.arange(len(n)), torch.tensor(n)).to(q.device)
+    mask = (scale_of[None, :] == scale_of[:, None]) | (scale_of[None, :] == scale_of[:, None] - 1)
+    qq, kk, vv = (t.detach().clone().requires_grad_(True) for t in (q, k, v))
+
+    def step():
+        out = F.scaled_dot_product_attention(qq, kk, vv, attn_mask=mask, scale=wl.softmax_scale)
+        out.backward(do)
+        qq.grad = kk.grad = vv.grad = None
+
+    step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        step()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def time_scale_steps(hmar, wl_inf, dev, reps=5):
+    """ms per inference step of every scale of the 512x512 d24 inference sweep (B=64, H=24; each step is
+    one masked sub-step: fresh Q and own-scale K/V, the previous scale's K/V kept)."""
+    import torch
+    from workloads.device import bulk_normal
+    out = []
+    for s, side in enumerate(wl_inf.side_lens):
+        side_prev = wl_inf.side_lens[s - 1] if s else 0
+        t = [bulk_normal(wl_inf.seed + s, i, wl_inf.B, wl_inf.H, (side_prev if i in (1, 2) else side) ** 2, wl_inf.D,
+                         torch.bfloat16, dev) if (s or i not in (1, 2)) else None for i in range(5)]
+        o = torch.empty_like(t[0])
+        for _ in range(2):
+            hmar.hmar_attn_scale_step(*t, side_prev, side, wl_inf.softmax_scale, out=o, want_lse=False)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            hmar.hmar_attn_scale_step(*t, side_prev, side, wl_inf.softmax_scale, out=o, want_lse=False)
+        e1.record()
+        torch.cuda.synchronize()
+        out.append(round(e0.elapsed_time(e1) / reps, 4))
+    return out
+
+
 def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -213,6 +263,24 @@ def run_ours(args, wl):
     if status != 0:
         raise RuntimeError(f"device status {status} detail {detail:#x}")
 
+    # ---- context legs, outside the timed region (rank 0 only): dense masked comparison, inference sweep
+    extras = {}
+    if rank == 0 and not args.no_extras:
+        try:
+            dense_ms = time_dense_masked(wl, q, k, v, do)
+            extras["dense_masked_sdpa"] = {"ms_fwd_bwd": dense_ms, "speedup_over_it": dense_ms / (total_ms / args.steps),
+                                           "what": "torch SDPA with the explicit boolean mask, same shape, same GPU"}
+        except Exception as e:     # the comparison is context; its failure must not lose the benchmark line
+            extras["dense_masked_sdpa"] = {"error": str(e)[:200]}
+        torch.cuda.empty_cache()
+        if args.batch == 0:
+            from workloads import CONFIGS
+            ms = time_scale_steps(hmar, CONFIGS["512_d24_infer"], dev)
+            extras["scale_step_ms"] = {"workload": "512_d24_infer, B=64 H=24, one sub-step per call", "per_scale": ms,
+                                       "sweep_4_sub_steps": round(4 * sum(ms), 4)}
+            torch.cuda.empty_cache()
+    args.extras = extras
+
     # ---- end to end: pinned host tensors in, results back to the host, inside the timed region
     if args.no_e2e:
         return _finish(args, wl, world, rank, dev, total_ms, float("nan"), fwd_ms, bwd_ms, launches, clocks, kernels)
@@ -293,6 +361,7 @@ def _finish(args, wl, world, rank, dev, total_ms, e2e_ms, fwd_ms, bwd_ms, launch
             "gpu_launches": int(launches),
             "clocks": clocks,
         }
+        line.update(getattr(args, "extras", {}))
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -308,6 +377,7 @@ def main():
                     help="override the batch size (profiling on a reduced case; named in config.workload)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
+    ap.add_argument("--no-extras", action="store_true", help="skip the dense masked comparison and the inference sweep")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     from workloads import CONFIGS

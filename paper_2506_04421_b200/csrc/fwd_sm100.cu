@@ -337,14 +337,14 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     if (!(col0 + 32 + i >= c_lo && col0 + 32 + i < c_hi)) b1[i] = 0xff800000u;
                 }
             }
-            float mx = -INFINITY;
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};     // four chains of maxima, not one of 64
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(b0[i]));
+            for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(b0[i]));
             if (two) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(b1[i]));
+                for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(b1[i]));
             }
-            mx *= sl2;                                          // softmax_scale > 0
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;     // softmax_scale > 0
 
             // Keep the running maximum unless this tile exceeds it by more than the threshold.  O_h is
             // quiet here: the product that precedes S_h of this tile in the tensor core's queue is the
