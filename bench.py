@@ -31,7 +31,8 @@ UNIT = "TFLOP/s"
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
-NCU_TRAFFIC_BYTES = {"hmar_bwd": None, "hmar_fwd": None}
+# The captures are of the batch-4 case (traffic grows in proportion to the heads), scaled by 4 to the full batch.
+NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (234_533_632 + 113_963_264), "hmar_fwd": 4 * (82_637_312 + 11_088_128)}
 
 
 def pairs_per_head(side_lens):
@@ -353,7 +354,8 @@ def _finish(args, wl, world, rank, dev, total_ms, e2e_ms, fwd_ms, bwd_ms, launch
             "roofline": {"bound": "tensor", "kernel": dom, "achieved": dom_tf, "peak": peaks["bf16_tflops"],
                          "unit": "TFLOP/s", "frac": dom_tf / peaks["bf16_tflops"],
                          "peak_source": peaks["source"] + " burst", "avg_launch_ms": dom_ms,
-                         "algorithmic_flops_per_launch": f_bwd, "traffic": NCU_TRAFFIC_BYTES["hmar_bwd"]},
+                         "algorithmic_flops_per_launch": f_bwd,
+                         "traffic": NCU_TRAFFIC_BYTES["hmar_bwd"] * B // 16},
             "kernels": per_kernel,
             "cpu_baseline": cpu_base,
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
