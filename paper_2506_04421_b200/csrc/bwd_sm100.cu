@@ -120,54 +120,59 @@ __device__ __forceinline__ void load_swizzled_row(const uint8_t* tile, int r, ui
     }
 }
 
-// One key row, 32 query columns (chunk c of the half that starts at column cbase of the step):
-// P^T = 2^(S^T * scale * log2e - lse * log2e) and dS^T = P^T o (dP^T - delta) in fp32.  P^T (bf16) goes back to
-// TMEM over S^T and dS^T (bf16) over dP^T - the 16 packed columns of chunk c start at column c * 16 of the
-// half, which this thread has already read - and dS^T also goes to shared memory (4 pieces of 8 queries,
-// 128-byte swizzle on the key row j).  MASKED: only columns [c_lo, c_hi) of the step are visible to this row.
+// The 64 query columns of one half step for the 32 key rows of one warp:
+// P^T = 2^(S^T * scale * log2e - lse * log2e) and dS^T = P^T o (dP^T - delta) in fp32.
+// S^T and dP^T are read 16 key rows at a time in the layout in which a thread holds, of two rows, the
+// column pairs 8k + 2(t % 4) + {0, 1}: a thread then needs lse and delta of 16 columns only (eight 8-byte
+// loads each, one shared-memory wavefront per load; one key row per thread would need all 64 columns as
+// broadcast loads, which were the largest share of the shared-memory traffic of the LSU).  A column pair
+// packs into one bf16x2: P^T goes back to TMEM over S^T and dS^T over dP^T with the matching store layout
+// (the 32 packed columns start at the half's first column, which this warp has already read for these
+// rows), and dS^T also goes to shared memory, 4 bytes per pair (a warp's store covers 16 bytes of 8 rows,
+// 128-byte swizzle on the key row: no bank conflicts).
+// MASKED: row i of this thread's four rows sees only columns [c_lo[i], c_hi[i]) of the step.
 template <bool MASKED>
-__device__ __forceinline__ void softmax_grad_chunk(uint32_t lane_base, int cbase, int c, const float* lse2, const float* delta,
-                                                   float sl2, int c_lo, int c_hi, uint8_t* ds_row, int j) {
-    const int c0 = cbase + c * 32;          // first query column of the chunk inside the step
-    uint32_t s_buf[32], dp_buf[32];
-    tmem_ld32(lane_base + COL_ST + c0, s_buf);
-    tmem_ld32(lane_base + COL_DPT + c0, dp_buf);
-    // lse / delta of the chunk's 32 queries while the TMEM loads are in flight
-    float4 ls[8], de[8];
-    const float4* lse4 = reinterpret_cast<const float4*>(lse2 + c0);
-    const float4* del4 = reinterpret_cast<const float4*>(delta + c0);
+__device__ __forceinline__ void softmax_grad_half(uint32_t lane_base, int cbase, const float* lse2, const float* delta,
+                                                  float sl2, const int (&c_lo)[4], const int (&c_hi)[4], uint8_t* ds_tile,
+                                                  int quarter, int lane) {
+    const int tq = lane & 3, tr = lane >> 2;
+    float2 ls[8], de[8];
 #pragma unroll
-    for (int t = 0; t < 8; ++t) { ls[t] = lse4[t]; de[t] = del4[t]; }
-    tmem_ld_wait();
-    uint32_t p_pack[16], ds_pack[16];
-#pragma unroll
-    for (int t = 0; t < 32; t += 4) {
-        float p0 = ex2(fmaf(__uint_as_float(s_buf[t]), sl2, -ls[t / 4].x));
-        float p1 = ex2(fmaf(__uint_as_float(s_buf[t + 1]), sl2, -ls[t / 4].y));
-        float p2 = ex2(fmaf(__uint_as_float(s_buf[t + 2]), sl2, -ls[t / 4].z));
-        float p3 = ex2(fmaf(__uint_as_float(s_buf[t + 3]), sl2, -ls[t / 4].w));
-        if (MASKED) {
-            p0 = (c0 + t >= c_lo && c0 + t < c_hi) ? p0 : 0.f;
-            p1 = (c0 + t + 1 >= c_lo && c0 + t + 1 < c_hi) ? p1 : 0.f;
-            p2 = (c0 + t + 2 >= c_lo && c0 + t + 2 < c_hi) ? p2 : 0.f;
-            p3 = (c0 + t + 3 >= c_lo && c0 + t + 3 < c_hi) ? p3 : 0.f;
-        }
-        const float d0 = p0 * (__uint_as_float(dp_buf[t]) - de[t / 4].x);
-        const float d1 = p1 * (__uint_as_float(dp_buf[t + 1]) - de[t / 4].y);
-        const float d2 = p2 * (__uint_as_float(dp_buf[t + 2]) - de[t / 4].z);
-        const float d3 = p3 * (__uint_as_float(dp_buf[t + 3]) - de[t / 4].w);
-        p_pack[t / 2] = pack_bf16(p0, p1);
-        p_pack[t / 2 + 1] = pack_bf16(p2, p3);
-        ds_pack[t / 2] = pack_bf16(d0, d1);
-        ds_pack[t / 2 + 1] = pack_bf16(d2, d3);
+    for (int k = 0; k < 8; ++k) {
+        ls[k] = *reinterpret_cast<const float2*>(lse2 + cbase + 8 * k + 2 * tq);
+        de[k] = *reinterpret_cast<const float2*>(delta + cbase + 8 * k + 2 * tq);
     }
-    tmem_st16(lane_base + COL_ST + cbase + c * 16, p_pack);
-    tmem_st16(lane_base + COL_DPT + cbase + c * 16, ds_pack);
 #pragma unroll
-    for (int ch = 0; ch < 4; ++ch) {
-        const int piece = c * 4 + ch;
-        const uint4 val = make_uint4(ds_pack[4 * ch], ds_pack[4 * ch + 1], ds_pack[4 * ch + 2], ds_pack[4 * ch + 3]);
-        *reinterpret_cast<uint4*>(ds_row + ((piece ^ (j & 7)) << 4)) = val;
+    for (int hl = 0; hl < 2; ++hl) {                    // lanes 0-15, then 16-31 of the warp's quarter
+        const uint32_t taddr = lane_base + ((uint32_t)(hl * 16) << 16);
+        uint32_t s_buf[32], dp_buf[32];
+        tmem_ld_16x256b_x8(taddr + COL_ST + cbase, s_buf);
+        tmem_ld_16x256b_x8(taddr + COL_DPT + cbase, dp_buf);
+        tmem_ld_wait();
+        uint32_t p_pack[16], ds_pack[16];
+        // key rows of this thread: quarter * 32 + hl * 16 + tr (+ 8); both have (row & 7) == tr
+        uint8_t* ds_row = ds_tile + (quarter * 4 + hl * 2) * 1024 + tr * 128 + tq * 4;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+#pragma unroll
+            for (int rs = 0; rs < 2; ++rs) {
+                float p0 = ex2(fmaf(__uint_as_float(s_buf[4 * k + 2 * rs]), sl2, -ls[k].x));
+                float p1 = ex2(fmaf(__uint_as_float(s_buf[4 * k + 2 * rs + 1]), sl2, -ls[k].y));
+                if (MASKED) {
+                    const int c = cbase + 8 * k + 2 * tq, i = hl * 2 + rs;
+                    p0 = (c >= c_lo[i] && c < c_hi[i]) ? p0 : 0.f;
+                    p1 = (c + 1 >= c_lo[i] && c + 1 < c_hi[i]) ? p1 : 0.f;
+                }
+                const float d0 = p0 * (__uint_as_float(dp_buf[4 * k + 2 * rs]) - de[k].x);
+                const float d1 = p1 * (__uint_as_float(dp_buf[4 * k + 2 * rs + 1]) - de[k].y);
+                p_pack[2 * k + rs] = pack_bf16(p0, p1);
+                ds_pack[2 * k + rs] = pack_bf16(d0, d1);
+                // 8-row groups are 1024 bytes apart; 16-byte piece k of a row sits at position k ^ (row & 7)
+                *reinterpret_cast<uint32_t*>(ds_row + rs * 1024 + ((k ^ tr) << 4)) = ds_pack[2 * k + rs];
+            }
+        }
+        tmem_st_16x128b_x8(taddr + COL_ST + cbase, p_pack);
+        tmem_st_16x128b_x8(taddr + COL_DPT + cbase, ds_pack);
     }
 }
 
@@ -520,7 +525,6 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const int j = quarter * 32 + lane;                  // key row inside the tile
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
         const float sl2 = args.scale_log2;
-        const int ds_row_off = (j >> 3) * 1024 + (j & 7) * 128;
         uint32_t s_buf[32], dp_buf[32];                     // K / V row on its way to TMEM; dK / dV row at the end of an item
         bool ok = true;
         int gs = 0;                                         // steps seen so far (aux ring, dS buffer parity)
@@ -531,14 +535,23 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             const BwdWork w = get_work(g);
             const int n_steps = steps_of(w);
             const int item = g - item_begin;
-            const bool row_ok = j < w.row_count;
-            int qlo = w.q_begin, qhi = w.q_end;             // queries that may see this key row
-            if (!w.uniform && row_ok) {
-                const int s = scale_of_row(args.st, w.row_begin + j);
-                qlo = args.st.start[s];
-                qhi = args.st.start[min(s + 2, args.st.n_scales)];
-            }
+            const bool row_ok = j < w.row_count;            // this thread's row in the 32x32b layout (K / V copy, dK / dV)
+            // the four key rows this thread works on in the softmax-gradient layout, and the queries that may see them
             const bool tile_masked = (!w.uniform) || (w.row_count < BKV);
+            int qlo[4], qhi[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int rr = quarter * 32 + (i >> 1) * 16 + (lane >> 2) + (i & 1) * 8;
+                qlo[i] = w.q_begin; qhi[i] = w.q_end;
+                if (tile_masked) {
+                    if (rr >= w.row_count) { qlo[i] = 0; qhi[i] = 0; }
+                    else if (!w.uniform) {
+                        const int sc = scale_of_row(args.st, w.row_begin + rr);
+                        qlo[i] = args.st.start[sc];
+                        qhi[i] = args.st.start[min(sc + 2, args.st.n_scales)];
+                    }
+                }
+            }
 
             // ---- K (warpgroup 0) / V (warpgroup 1) row to TMEM: A operands of S^T = K Q^T and dP^T = V dO^T
             ok = __all_sync(0xffffffffu, mbar_wait(&sm.kv_full, item & 1, abort_flag));
@@ -554,9 +567,6 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 const int n_valid = min(BQ, w.q_end - q0);
                 const int n_cols = half_cols(w, i, h);
                 const int cbase = h * HQ;                   // first query column of this half inside the step
-                // visible query columns of this key row in this step: [c_lo, c_hi)
-                const int c_lo = row_ok ? max(qlo - q0, 0) : 0;
-                const int c_hi = row_ok ? min(qhi - q0, n_valid) : 0;
 
                 const int aslot = gs % AUX_STAGES;
                 ok = __all_sync(0xffffffffu, mbar_wait(&sm.aux_full[aslot], (gs / AUX_STAGES) & 1, abort_flag));
@@ -567,16 +577,20 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     if (!ok) { if (lane == 0) report_timeout(args.status, 0x1580 + i); break; }
                     ++nsh;
                     tc_fence_after();
-                    uint8_t* ds_row = sm.ds[gs & 1][h] + ds_row_off;
-                    // 32 query columns at a time; tiles whose rows all see every column skip the mask code
+                    // tiles whose rows all see every column skip the mask code
+                    if (tile_masked) {
+                        int c_lo[4], c_hi[4];               // visible query columns of the four rows in this step
 #pragma unroll
-                    for (int c = 0; c < 2; ++c) {
-                        if (c * 32 < n_cols) {
-                            if (tile_masked)
-                                softmax_grad_chunk<true>(lane_base, cbase, c, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi, ds_row, j);
-                            else
-                                softmax_grad_chunk<false>(lane_base, cbase, c, sm.lse2[aslot], sm.delta[aslot], sl2, 0, 0, ds_row, j);
+                        for (int r4 = 0; r4 < 4; ++r4) {
+                            c_lo[r4] = max(qlo[r4] - q0, 0);
+                            c_hi[r4] = min(qhi[r4] - q0, n_valid);
                         }
+                        softmax_grad_half<true>(lane_base, cbase, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi,
+                                                sm.ds[gs & 1][h], quarter, lane);
+                    } else {
+                        const int none[4] = {0, 0, 0, 0};
+                        softmax_grad_half<false>(lane_base, cbase, sm.lse2[aslot], sm.delta[aslot], sl2, none, none,
+                                                 sm.ds[gs & 1][h], quarter, lane);
                     }
                     tmem_st_wait();
                     tc_fence_before();
