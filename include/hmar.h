@@ -49,6 +49,16 @@ typedef enum {
 
 #define HMAR_MAX_SCALES 64
 
+/* Which scales a token of scale k attends to.  All three are block masks over the same flattened
+ * sequence in which the allowed keys of a query are one contiguous range, so one scheduler and one set
+ * of kernels serves them.
+ *   HMAR_WINDOW_MARKOV : scales k-1 and k - HMAR's Markovian mask (Sec. 4.1, Fig. attn-mask); what the
+ *                        entry points without `_window` compute.
+ *   HMAR_WINDOW_CAUSAL : scales 1..k - VAR's block-causal mask (Sec. 3, Fig. attn-mask), the workload the
+ *                        paper's attention benchmark compares against (App. B.4).
+ *   HMAR_WINDOW_SELF   : scale k only - the literal "block-diagonal" reading of Sec. 1 / App. B.3. */
+typedef enum { HMAR_WINDOW_MARKOV = 0, HMAR_WINDOW_CAUSAL = 1, HMAR_WINDOW_SELF = 2 } hmar_window;
+
 /* Training forward (Sec. 4.1; App. B.4 benchmarks this pass).
  *   q, k, v : [B,H,L,D] in;  out : [B,H,L,D] out;  lse : [B,H,L] fp32 out.
  *   side_lens : host array of n_scales positive side lengths (any order of sizes is accepted). */
@@ -58,6 +68,16 @@ int hmar_attn_fwd(const void* q, const void* k, const void* v, void* out, float*
 int hmar_attn_fwd_f32(const float* q, const float* k, const float* v, float* out, float* lse,
                       int B, int H, int D, int n_scales, const int* side_lens,
                       float softmax_scale, void* stream);
+
+/* The same forward under another block mask of the same family (see hmar_window).  Everything else -
+ * layouts, lse convention, precision, errors - is as for hmar_attn_fwd; an unknown `window` is
+ * HMAR_ERR_BAD_ARG. */
+int hmar_attn_fwd_window(const void* q, const void* k, const void* v, void* out, float* lse,
+                         int B, int H, int D, int n_scales, const int* side_lens, int window,
+                         float softmax_scale, void* stream);
+int hmar_attn_fwd_window_f32(const float* q, const float* k, const float* v, float* out, float* lse,
+                             int B, int H, int D, int n_scales, const int* side_lens, int window,
+                             float softmax_scale, void* stream);
 
 /* Bytes of caller-provided device scratch the backward needs for this problem (0 on bad arguments).
  * The scratch holds delta = rowsum(dO o O) and the fp32 dQ accumulator; its contents on entry do not
@@ -79,6 +99,19 @@ int hmar_attn_bwd_f32(const float* q, const float* k, const float* v, const floa
                       void* workspace, size_t workspace_bytes,
                       int B, int H, int D, int n_scales, const int* side_lens,
                       float softmax_scale, void* stream);
+
+/* The same backward under another block mask of the same family (see hmar_window); `lse` and `out` must
+ * come from hmar_attn_fwd_window with the same `window`.  Workspace as for hmar_attn_bwd. */
+int hmar_attn_bwd_window(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                         const void* dout, void* dq, void* dk, void* dv,
+                         void* workspace, size_t workspace_bytes,
+                         int B, int H, int D, int n_scales, const int* side_lens, int window,
+                         float softmax_scale, void* stream);
+int hmar_attn_bwd_window_f32(const float* q, const float* k, const float* v, const float* out, const float* lse,
+                             const float* dout, float* dq, float* dk, float* dv,
+                             void* workspace, size_t workspace_bytes,
+                             int B, int H, int D, int n_scales, const int* side_lens, int window,
+                             float softmax_scale, void* stream);
 
 /* Backward for callers that cannot allocate device memory (the paper has no counterpart; this is a
  * library convenience).  Same inputs, outputs and arithmetic as hmar_attn_bwd (bf16), but no workspace
@@ -129,6 +162,9 @@ int hmar_attn_scale_step_f32(const float* q, const float* k_prev, const float* v
  * hmar_status; writes at most max_tiles entries (pass NULL / 0 to query the count).  Host only. */
 int hmar_schedule_tiles(int n_scales, const int* side_lens, int direction,
                         int32_t* tiles, int max_tiles);
+/* The same for any mask of the family (see hmar_window). */
+int hmar_schedule_tiles_window(int n_scales, const int* side_lens, int window, int direction,
+                               int32_t* tiles, int max_tiles);
 
 /* Blocks until the work queued on the current device has finished, then returns the code recorded
  * by the kernels since the last call (HMAR_OK, or HMAR_ERR_DEVICE_TIMEOUT with *detail, if not NULL,

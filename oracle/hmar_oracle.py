@@ -64,9 +64,27 @@ def block_causal_mask(side_lens):
     return s[None, :] <= s[:, None]
 
 
-def count_pairs(side_lens):
-    """Number of unmasked (i, j) pairs per head under the HMAR mask."""
-    return int(hmar_mask(side_lens).sum())
+def block_diagonal_mask(side_lens):
+    """Scale k attends to scale k only: the literal block-diagonal pattern of Sec. 1 / App. B.3."""
+    s = scale_of_token(side_lens)
+    return s[None, :] == s[:, None]
+
+
+def window_mask(side_lens, window="markov"):
+    """The mask of the family named by `window`: "markov" (HMAR, scales k-1 and k), "causal" (VAR's
+    block-causal mask, Sec. 3) or "self" (block-diagonal)."""
+    if window == "markov":
+        return hmar_mask(side_lens)
+    if window == "causal":
+        return block_causal_mask(side_lens)
+    if window == "self":
+        return block_diagonal_mask(side_lens)
+    raise ValueError("window must be 'markov', 'causal' or 'self'")
+
+
+def count_pairs(side_lens, window="markov"):
+    """Number of unmasked (i, j) pairs per head under the mask."""
+    return int(window_mask(side_lens, window).sum())
 
 
 def _masked_softmax(S, M):
@@ -88,20 +106,20 @@ def attention_probs(q, k, mask, softmax_scale):
     return _masked_softmax(S, mask)
 
 
-def attn_fwd(q, k, v, side_lens, softmax_scale):
+def attn_fwd(q, k, v, side_lens, softmax_scale, window="markov"):
     """Training forward. q, k, v: [..., L, D]. Returns out [..., L, D], lse [..., L] (float64).
 
     lse_i = ln sum_j exp(softmax_scale * q_i . k_j) over the allowed j.
     """
     v = np.asarray(v, dtype=np.float64)
-    M = hmar_mask(side_lens)
+    M = window_mask(side_lens, window)
     if q.shape[-2] != M.shape[0]:
         raise ValueError("sequence length does not match side_lens")
     P, lse = attention_probs(q, k, M, softmax_scale)
     return P @ v, lse
 
 
-def attn_bwd(q, k, v, dout, side_lens, softmax_scale):
+def attn_bwd(q, k, v, dout, side_lens, softmax_scale, window="markov"):
     """Training backward: gradients of sum(out * dout) w.r.t. q, k, v (float64).
 
     dV = P^T dO;  dP = dO V^T;  delta_i = sum_j P_ij dP_ij;  dS = P o (dP - delta);
@@ -111,7 +129,7 @@ def attn_bwd(q, k, v, dout, side_lens, softmax_scale):
     k = np.asarray(k, dtype=np.float64)
     v = np.asarray(v, dtype=np.float64)
     dout = np.asarray(dout, dtype=np.float64)
-    M = hmar_mask(side_lens)
+    M = window_mask(side_lens, window)
     P, _ = attention_probs(q, k, M, softmax_scale)
     dV = np.swapaxes(P, -1, -2) @ dout
     dP = dout @ np.swapaxes(v, -1, -2)

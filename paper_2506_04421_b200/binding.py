@@ -21,9 +21,14 @@ HMAR_ERR_CUDA = -3
 HMAR_ERR_WORKSPACE = -4
 HMAR_ERR_DEVICE_TIMEOUT = -5
 
+HMAR_WINDOW_MARKOV = 0      # scales k-1 and k (HMAR)
+HMAR_WINDOW_CAUSAL = 1      # scales 1..k (VAR's block-causal mask)
+HMAR_WINDOW_SELF = 2        # scale k only (block-diagonal)
+
 EXPORTED_SYMBOLS = (
-    "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd",
-    "hmar_attn_bwd_f32", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_schedule_tiles",
+    "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_fwd_window", "hmar_attn_fwd_window_f32",
+    "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd", "hmar_attn_bwd_f32", "hmar_attn_bwd_window",
+    "hmar_attn_bwd_window_f32", "hmar_schedule_tiles_window", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_schedule_tiles",
     "hmar_device_status", "hmar_profile_begin", "hmar_profile_end", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
     "hmar_status_string",
 )
@@ -48,10 +53,15 @@ def lib():
     i = ctypes.c_int
     L.hmar_attn_fwd.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, ip, fp, vp]
     L.hmar_attn_fwd_f32.argtypes = L.hmar_attn_fwd.argtypes
+    L.hmar_attn_fwd_window.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, ip, i, fp, vp]
+    L.hmar_attn_fwd_window_f32.argtypes = L.hmar_attn_fwd_window.argtypes
     L.hmar_attn_bwd_workspace_bytes.argtypes = [i, i, i, i, ip]
     L.hmar_attn_bwd_workspace_bytes.restype = ctypes.c_size_t
     L.hmar_attn_bwd.argtypes = [vp] * 9 + [vp, ctypes.c_size_t, i, i, i, i, ip, fp, vp]
     L.hmar_attn_bwd_f32.argtypes = L.hmar_attn_bwd.argtypes
+    L.hmar_attn_bwd_window.argtypes = [vp] * 9 + [vp, ctypes.c_size_t, i, i, i, i, ip, i, fp, vp]
+    L.hmar_attn_bwd_window_f32.argtypes = L.hmar_attn_bwd_window.argtypes
+    L.hmar_schedule_tiles_window.argtypes = [i, ip, i, i, ctypes.POINTER(ctypes.c_int32), i]
     L.hmar_attn_bwd_noalloc.argtypes = [vp] * 9 + [i, i, i, i, ip, fp, vp]
     L.hmar_attn_scale_step.argtypes = [vp] * 7 + [i, i, i, i, i, fp, vp]
     L.hmar_attn_scale_step_f32.argtypes = L.hmar_attn_scale_step.argtypes
@@ -109,8 +119,9 @@ def _need(*tensors):
             raise ValueError("tensors must be contiguous CUDA tensors")
 
 
-def hmar_attn_fwd(q, k, v, side_lens, softmax_scale, out=None, lse=None, stream=None):
-    """Training forward. q, k, v: [B,H,L,D]. Returns (out [B,H,L,D], lse [B,H,L] fp32)."""
+def hmar_attn_fwd(q, k, v, side_lens, softmax_scale, out=None, lse=None, stream=None, window=HMAR_WINDOW_MARKOV):
+    """Training forward. q, k, v: [B,H,L,D]. Returns (out [B,H,L,D], lse [B,H,L] fp32).
+    `window` other than HMAR_WINDOW_MARKOV goes through hmar_attn_fwd_window."""
     _need(q, k, v, out, lse)
     B, H, L, D = q.shape
     if out is None:
@@ -118,6 +129,11 @@ def hmar_attn_fwd(q, k, v, side_lens, softmax_scale, out=None, lse=None, stream=
     if lse is None:
         lse = torch.empty((B, H, L), dtype=torch.float32, device=q.device)
     sides, n = _sides(side_lens)
+    if window != HMAR_WINDOW_MARKOV:
+        fn = lib().hmar_attn_fwd_window_f32 if _is_f32(q) else lib().hmar_attn_fwd_window
+        _check(fn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, D, n, sides, int(window),
+                  float(softmax_scale), _stream(stream)), "hmar_attn_fwd_window")
+        return out, lse
     fn = lib().hmar_attn_fwd_f32 if _is_f32(q) else lib().hmar_attn_fwd
     _check(fn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, D, n, sides,
               float(softmax_scale), _stream(stream)), "hmar_attn_fwd")
@@ -130,8 +146,9 @@ def hmar_attn_bwd_workspace_bytes(B, H, D, side_lens):
 
 
 def hmar_attn_bwd(q, k, v, out, lse, dout, side_lens, softmax_scale, dq=None, dk=None, dv=None,
-                  workspace=None, stream=None):
-    """Training backward. Returns (dq, dk, dv), each [B,H,L,D]."""
+                  workspace=None, stream=None, window=HMAR_WINDOW_MARKOV):
+    """Training backward. Returns (dq, dk, dv), each [B,H,L,D].
+    `window` other than HMAR_WINDOW_MARKOV goes through hmar_attn_bwd_window."""
     _need(q, k, v, out, lse, dout, dq, dk, dv, workspace)
     B, H, L, D = q.shape
     dq = torch.empty_like(q) if dq is None else dq
@@ -141,6 +158,12 @@ def hmar_attn_bwd(q, k, v, out, lse, dout, side_lens, softmax_scale, dq=None, dk
         workspace = torch.empty(hmar_attn_bwd_workspace_bytes(B, H, D, side_lens), dtype=torch.uint8,
                                 device=q.device)
     sides, n = _sides(side_lens)
+    if window != HMAR_WINDOW_MARKOV:
+        fn = lib().hmar_attn_bwd_window_f32 if _is_f32(q) else lib().hmar_attn_bwd_window
+        _check(fn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv),
+                  _ptr(workspace), workspace.numel() * workspace.element_size(), B, H, D, n, sides, int(window),
+                  float(softmax_scale), _stream(stream)), "hmar_attn_bwd_window")
+        return dq, dk, dv
     fn = lib().hmar_attn_bwd_f32 if _is_f32(q) else lib().hmar_attn_bwd
     _check(fn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout), _ptr(dq), _ptr(dk), _ptr(dv),
               _ptr(workspace), workspace.numel() * workspace.element_size(), B, H, D, n, sides,
@@ -184,14 +207,14 @@ def hmar_attn_scale_step(q, k_prev, v_prev, k_cur, v_cur, side_prev, side_cur, s
     return out, lse
 
 
-def hmar_schedule_tiles(side_lens, direction):
+def hmar_schedule_tiles(side_lens, direction, window=HMAR_WINDOW_MARKOV):
     """Work list of one head as a list of dicts (host only; needs no GPU)."""
     sides, n = _sides(side_lens)
-    count = lib().hmar_schedule_tiles(n, sides, int(direction), None, 0)
+    count = lib().hmar_schedule_tiles_window(n, sides, int(window), int(direction), None, 0)
     if count < 0:
         raise HmarError(count, "hmar_schedule_tiles")
     buf = (ctypes.c_int32 * (6 * count))()
-    lib().hmar_schedule_tiles(n, sides, int(direction), buf, count)
+    lib().hmar_schedule_tiles_window(n, sides, int(window), int(direction), buf, count)
     keys = ("row_begin", "row_count", "partner_begin", "partner_end", "uniform", "cost")
     return [dict(zip(keys, buf[6 * t:6 * t + 6])) for t in range(count)]
 

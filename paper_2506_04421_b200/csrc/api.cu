@@ -65,15 +65,16 @@ static int check_shape(int B, int H, int D) {
     return HMAR_OK;
 }
 
-static int check_sides(int n_scales, const int* side_lens, ScaleTable* st) {
+static int check_sides(int n_scales, const int* side_lens, int window, ScaleTable* st) {
     if (n_scales <= 0 || n_scales > HMAR_MAX_SCALES || side_lens == nullptr) return HMAR_ERR_BAD_ARG;
+    if (window != HMAR_WINDOW_MARKOV && window != HMAR_WINDOW_CAUSAL && window != HMAR_WINDOW_SELF) return HMAR_ERR_BAD_ARG;
     long long total = 0;
     for (int s = 0; s < n_scales; ++s) {
         if (side_lens[s] <= 0 || side_lens[s] > 4096) return HMAR_ERR_BAD_ARG;
         total += (long long)side_lens[s] * side_lens[s];
     }
     if (total > (1 << 24)) return HMAR_ERR_BAD_ARG;
-    build_scale_table(n_scales, side_lens, st);
+    build_scale_table(n_scales, side_lens, window, st);
     return HMAR_OK;
 }
 
@@ -108,11 +109,11 @@ static int* device_status_ptr() {
 // ------------------------------------------------------------------------------------------------
 template <typename T>
 static int fwd_impl(const T* q, const T* k, const T* v, T* out, float* lse, int B, int H, int D,
-                    int n_scales, const int* side_lens, float softmax_scale, void* stream, bool tensor_core) {
+                    int n_scales, const int* side_lens, int window, float softmax_scale, void* stream, bool tensor_core) {
     int rc = check_shape(B, H, D);
     if (rc != HMAR_OK) return rc;
     ScaleTable st;
-    rc = check_sides(n_scales, side_lens, &st);
+    rc = check_sides(n_scales, side_lens, window, &st);
     if (rc != HMAR_OK) return rc;
     if (check_scale(softmax_scale) != HMAR_OK) return HMAR_ERR_BAD_ARG;
     if (!q || !k || !v || !out || !lse) return HMAR_ERR_BAD_ARG;
@@ -131,11 +132,11 @@ static int fwd_impl(const T* q, const T* k, const T* v, T* out, float* lse, int 
 template <typename T>
 static int bwd_impl(const T* q, const T* k, const T* v, const T* out, const float* lse, const T* dout,
                     T* dq, T* dk, T* dv, void* workspace, size_t workspace_bytes, int B, int H, int D,
-                    int n_scales, const int* side_lens, float softmax_scale, void* stream, bool tensor_core) {
+                    int n_scales, const int* side_lens, int window, float softmax_scale, void* stream, bool tensor_core) {
     int rc = check_shape(B, H, D);
     if (rc != HMAR_OK) return rc;
     ScaleTable st;
-    rc = check_sides(n_scales, side_lens, &st);
+    rc = check_sides(n_scales, side_lens, window, &st);
     if (rc != HMAR_OK) return rc;
     if (check_scale(softmax_scale) != HMAR_OK) return HMAR_ERR_BAD_ARG;
     if (!q || !k || !v || !out || !lse || !dout || !dq || !dk || !dv) return HMAR_ERR_BAD_ARG;
@@ -195,38 +196,64 @@ typedef __nv_bfloat16 bf16;
 
 extern "C" {
 
+int hmar_attn_fwd_window(const void* q, const void* k, const void* v, void* out, float* lse, int B, int H, int D,
+                         int n_scales, const int* side_lens, int window, float softmax_scale, void* stream) {
+    return fwd_impl<bf16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, lse, B, H, D, n_scales,
+                          side_lens, window, softmax_scale, stream, true);
+}
+
+int hmar_attn_fwd_window_f32(const float* q, const float* k, const float* v, float* out, float* lse, int B, int H,
+                             int D, int n_scales, const int* side_lens, int window, float softmax_scale, void* stream) {
+    return fwd_impl<float>(q, k, v, out, lse, B, H, D, n_scales, side_lens, window, softmax_scale, stream, false);
+}
+
 int hmar_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse, int B, int H, int D,
                   int n_scales, const int* side_lens, float softmax_scale, void* stream) {
-    return fwd_impl<bf16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (bf16*)out, lse, B, H, D, n_scales,
-                          side_lens, softmax_scale, stream, true);
+    return hmar_attn_fwd_window(q, k, v, out, lse, B, H, D, n_scales, side_lens, HMAR_WINDOW_MARKOV, softmax_scale, stream);
 }
 
 int hmar_attn_fwd_f32(const float* q, const float* k, const float* v, float* out, float* lse, int B, int H,
                       int D, int n_scales, const int* side_lens, float softmax_scale, void* stream) {
-    return fwd_impl<float>(q, k, v, out, lse, B, H, D, n_scales, side_lens, softmax_scale, stream, false);
+    return hmar_attn_fwd_window_f32(q, k, v, out, lse, B, H, D, n_scales, side_lens, HMAR_WINDOW_MARKOV, softmax_scale, stream);
 }
 
 size_t hmar_attn_bwd_workspace_bytes(int B, int H, int D, int n_scales, const int* side_lens) {
     ScaleTable st;
-    if (check_shape(B, H, D) != HMAR_OK || check_sides(n_scales, side_lens, &st) != HMAR_OK) return 0;
+    if (check_shape(B, H, D) != HMAR_OK || check_sides(n_scales, side_lens, HMAR_WINDOW_MARKOV, &st) != HMAR_OK) return 0;
     const size_t rows = (size_t)B * H * st.start[st.n_scales];
     return round256(rows * sizeof(float)) + round256(rows * kHeadDim * sizeof(float));
+}
+
+int hmar_attn_bwd_window(const void* q, const void* k, const void* v, const void* out, const float* lse,
+                         const void* dout, void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
+                         int B, int H, int D, int n_scales, const int* side_lens, int window, float softmax_scale,
+                         void* stream) {
+    return bwd_impl<bf16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (const bf16*)out, lse,
+                          (const bf16*)dout, (bf16*)dq, (bf16*)dk, (bf16*)dv, workspace, workspace_bytes, B, H,
+                          D, n_scales, side_lens, window, softmax_scale, stream, true);
+}
+
+int hmar_attn_bwd_window_f32(const float* q, const float* k, const float* v, const float* out, const float* lse,
+                             const float* dout, float* dq, float* dk, float* dv, void* workspace,
+                             size_t workspace_bytes, int B, int H, int D, int n_scales, const int* side_lens,
+                             int window, float softmax_scale, void* stream) {
+    return bwd_impl<float>(q, k, v, out, lse, dout, dq, dk, dv, workspace, workspace_bytes, B, H, D, n_scales,
+                           side_lens, window, softmax_scale, stream, false);
 }
 
 int hmar_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse,
                   const void* dout, void* dq, void* dk, void* dv, void* workspace, size_t workspace_bytes,
                   int B, int H, int D, int n_scales, const int* side_lens, float softmax_scale, void* stream) {
-    return bwd_impl<bf16>((const bf16*)q, (const bf16*)k, (const bf16*)v, (const bf16*)out, lse,
-                          (const bf16*)dout, (bf16*)dq, (bf16*)dk, (bf16*)dv, workspace, workspace_bytes, B, H,
-                          D, n_scales, side_lens, softmax_scale, stream, true);
+    return hmar_attn_bwd_window(q, k, v, out, lse, dout, dq, dk, dv, workspace, workspace_bytes, B, H, D, n_scales,
+                                side_lens, HMAR_WINDOW_MARKOV, softmax_scale, stream);
 }
 
 int hmar_attn_bwd_f32(const float* q, const float* k, const float* v, const float* out, const float* lse,
                       const float* dout, float* dq, float* dk, float* dv, void* workspace,
                       size_t workspace_bytes, int B, int H, int D, int n_scales, const int* side_lens,
                       float softmax_scale, void* stream) {
-    return bwd_impl<float>(q, k, v, out, lse, dout, dq, dk, dv, workspace, workspace_bytes, B, H, D, n_scales,
-                           side_lens, softmax_scale, stream, false);
+    return hmar_attn_bwd_window_f32(q, k, v, out, lse, dout, dq, dk, dv, workspace, workspace_bytes, B, H, D,
+                                    n_scales, side_lens, HMAR_WINDOW_MARKOV, softmax_scale, stream);
 }
 
 int hmar_attn_scale_step(const void* q, const void* k_prev, const void* v_prev, const void* k_cur,
@@ -245,8 +272,13 @@ int hmar_attn_scale_step_f32(const float* q, const float* k_prev, const float* v
 }
 
 int hmar_schedule_tiles(int n_scales, const int* side_lens, int direction, int32_t* tiles, int max_tiles) {
+    return hmar_schedule_tiles_window(n_scales, side_lens, HMAR_WINDOW_MARKOV, direction, tiles, max_tiles);
+}
+
+int hmar_schedule_tiles_window(int n_scales, const int* side_lens, int window, int direction, int32_t* tiles,
+                               int max_tiles) {
     ScaleTable st;
-    int rc = check_sides(n_scales, side_lens, &st);
+    int rc = check_sides(n_scales, side_lens, window, &st);
     if (rc != HMAR_OK) return rc;
     if (direction != 0 && direction != 1) return HMAR_ERR_BAD_ARG;
     std::vector<Tile> t = build_tiles(st, direction);

@@ -548,7 +548,7 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     else if (!w.uniform) {
                         const int sc = scale_of_row(args.st, w.row_begin + rr);
                         qlo[i] = args.st.start[sc];
-                        qhi[i] = args.st.start[min(sc + 2, args.st.n_scales)];
+                        qhi[i] = args.st.start[last_query_scale(args.st.window, sc, args.st.n_scales) + 1];
                     }
                 }
             }

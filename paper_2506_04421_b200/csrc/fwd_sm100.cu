@@ -297,7 +297,7 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         int lo = w.s0_begin, hi = w.s0_end;                    // per-row key bounds (training, packed tiles)
         if (!w.uniform && row_ok) {
             const int s = scale_of_row(args.st, row);
-            lo = args.st.start[s > 0 ? s - 1 : 0];
+            lo = args.st.start[first_key_scale(args.st.window, s)];
             hi = args.st.start[s + 1];
         }
         const float sl2 = args.scale_log2;

@@ -12,8 +12,23 @@ constexpr int kTileRows = 128;   // rows of one work tile (query rows forward, k
 // Offsets of the scales in the flattened sequence; passed to kernels by value.
 struct ScaleTable {
     int n_scales;
+    int window;                       // hmar_window: which scales a query of scale s sees
     int start[HMAR_MAX_SCALES + 1];   // start[n_scales] == L
 };
+
+#if defined(__CUDACC__)
+#define HMAR_HD __host__ __device__ __forceinline__
+#else
+#define HMAR_HD inline
+#endif
+// The keys a query of scale s sees are the scales first_key_scale(s) .. s, a contiguous range of the
+// flattened sequence; the queries that see a key of scale s are the scales s .. last_query_scale(s).
+HMAR_HD int first_key_scale(int window, int s) {
+    return window == HMAR_WINDOW_CAUSAL ? 0 : (window == HMAR_WINDOW_SELF ? s : (s > 0 ? s - 1 : 0));
+}
+HMAR_HD int last_query_scale(int window, int s, int n_scales) {
+    return window == HMAR_WINDOW_CAUSAL ? n_scales - 1 : (window == HMAR_WINDOW_SELF ? s : (s + 1 < n_scales ? s + 1 : s));
+}
 
 // One unit of work: `row_count` consecutive rows starting at `row_begin`, and the contiguous range
 // [partner_begin, partner_end) of the other operand those rows touch.
@@ -27,9 +42,9 @@ struct Tile {
     int32_t cost;      // number of kTileRows-wide partner tiles (for ordering)
 };
 
-// Forward bounds of query row `i` of scale s: keys [start[s-1], start[s+1]).
-// Backward bounds of key row `j` of scale s: queries [start[s], start[s+2]).
-void build_scale_table(int n_scales, const int* side_lens, ScaleTable* out);
+// Forward bounds of query row `i` of scale s: keys [start[first_key_scale(s)], start[s+1]).
+// Backward bounds of key row `j` of scale s: queries [start[s], start[last_query_scale(s)+1]).
+void build_scale_table(int n_scales, const int* side_lens, int window, ScaleTable* out);
 std::vector<Tile> build_tiles(const ScaleTable& st, int direction);
 
 #if defined(__CUDACC__)

@@ -77,7 +77,7 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
     if ((unsigned long long)L * B * H > kMaxRows) return HMAR_ERR_WORKSPACE;     // beyond the fixed scratch
 
     ScaleTable st;
-    build_scale_table(n_scales, side_lens, &st);
+    build_scale_table(n_scales, side_lens, HMAR_WINDOW_MARKOV, &st);
     const std::vector<Tile> tiles = build_tiles(st, 1);
     if (tiles.size() > kMaxWork) return HMAR_ERR_WORKSPACE;
 

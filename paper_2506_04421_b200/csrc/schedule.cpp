@@ -11,8 +11,9 @@
 
 namespace hmar {
 
-void build_scale_table(int n_scales, const int* side_lens, ScaleTable* out) {
+void build_scale_table(int n_scales, const int* side_lens, int window, ScaleTable* out) {
     out->n_scales = n_scales;
+    out->window = window;
     out->start[0] = 0;
     for (int s = 0; s < n_scales; ++s)
         out->start[s + 1] = out->start[s] + side_lens[s] * side_lens[s];
@@ -22,11 +23,11 @@ static void partner_range(const ScaleTable& st, int direction, int s_first, int 
                           int* begin, int* end) {
     const int K = st.n_scales;
     if (direction == 0) {           // queries of scales s_first..s_last -> keys
-        *begin = st.start[std::max(s_first - 1, 0)];
+        *begin = st.start[first_key_scale(st.window, s_first)];
         *end = st.start[s_last + 1];
     } else {                        // keys of scales s_first..s_last -> queries
         *begin = st.start[s_first];
-        *end = st.start[std::min(s_last + 2, K)];
+        *end = st.start[last_query_scale(st.window, s_last, K) + 1];
     }
 }
 

@@ -71,10 +71,10 @@ simt_fwd_kernel(const T* __restrict__ q, const T* __restrict__ k0, const T* __re
         hi = blk_hi = n0 + n1;
     } else {
         int s = scale_of_row(st, row);
-        lo = st.start[s > 0 ? s - 1 : 0];
+        lo = st.start[first_key_scale(st.window, s)];
         hi = st.start[s + 1];
         int sf = scale_of_row(st, row0), sl = scale_of_row(st, last_row);
-        blk_lo = st.start[sf > 0 ? sf - 1 : 0];
+        blk_lo = st.start[first_key_scale(st.window, sf)];
         blk_hi = st.start[sl + 1];
     }
 
@@ -157,9 +157,9 @@ simt_dq_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     const int row = row_ok ? row_raw : L - 1;
     const int last_row = min(row0 + ROWS, L) - 1;
     const int s_row = scale_of_row(st, row);
-    const int lo = st.start[s_row > 0 ? s_row - 1 : 0], hi = st.start[s_row + 1];
+    const int lo = st.start[first_key_scale(st.window, s_row)], hi = st.start[s_row + 1];
     const int sf = scale_of_row(st, row0), sl = scale_of_row(st, last_row);
-    const int blk_lo = st.start[sf > 0 ? sf - 1 : 0], blk_hi = st.start[sl + 1];
+    const int blk_lo = st.start[first_key_scale(st.window, sf)], blk_hi = st.start[sl + 1];
     const size_t head = (size_t)bh * L;
 
     float qr[DH], gr[DH], acc[DH];
@@ -223,9 +223,9 @@ simt_dkdv_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __re
     const int last_row = min(row0 + ROWS, L) - 1;
     const int K = st.n_scales;
     const int s_row = scale_of_row(st, row);
-    const int lo = st.start[s_row], hi = st.start[min(s_row + 2, K)];
+    const int lo = st.start[s_row], hi = st.start[last_query_scale(st.window, s_row, K) + 1];
     const int blk_lo = st.start[scale_of_row(st, row0)];
-    const int blk_hi = st.start[min(scale_of_row(st, last_row) + 2, K)];
+    const int blk_hi = st.start[last_query_scale(st.window, scale_of_row(st, last_row), K) + 1];
     const size_t head = (size_t)bh * L;
 
     float kr[DH], vr[DH], ak[DH], av[DH];

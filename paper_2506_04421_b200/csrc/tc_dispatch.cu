@@ -90,6 +90,7 @@ static const Plan* get_plan(const ScaleTable& st) {
     PlanKey key;
     if (cudaGetDevice(&key.device) != cudaSuccess) return nullptr;
     key.starts.assign(st.start, st.start + st.n_scales + 1);
+    key.starts.push_back(st.window);
     std::lock_guard<std::mutex> lock(g_plan_mu);
     auto it = g_plans.find(key);
     if (it != g_plans.end()) return &it->second;
@@ -199,6 +200,7 @@ int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const b
     a.lse = lse;
     a.status = status;
     a.st.n_scales = 0;
+    a.st.window = HMAR_WINDOW_MARKOV;
     return launch_fwd_tc(mq, mk0, mv0, mk1, mv1, a, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 

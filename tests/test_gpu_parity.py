@@ -110,6 +110,49 @@ def test_fp32_debug_build_512_shape_one_head():
     _run_training(_Wl(CONFIGS["512_d24_train"].side_lens, B=1, H=1), torch.float32)
 
 
+WINDOWS = [("causal", hmar.HMAR_WINDOW_CAUSAL), ("self", hmar.HMAR_WINDOW_SELF)]
+
+
+@pytest.mark.parametrize("window", WINDOWS, ids=[w[0] for w in WINDOWS])
+@pytest.mark.parametrize("sides", [(1, 2, 3, 4), (3, 11), (12, 11, 1), (2, 1, 3, 1, 2), (1, 2, 3, 4, 5, 6, 8, 10, 13, 16), (16, 3, 17)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_other_block_masks_fwd_bwd(sides, dtype, window):
+    """VAR's block-causal mask and the block-diagonal mask through the *_window entry points."""
+    wl = _Wl(sides)
+    is_f32 = dtype == torch.float32
+    q, k, v, do = training_inputs(wl, bf16=not is_f32)
+    tq, tk, tv, tdo = (to_device(x, wl.B, wl.H, dtype) for x in (q, k, v, do))
+    out, lse = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale, window=window[1])
+    ref_out, ref_lse = orc.attn_fwd(q, k, v, wl.side_lens, wl.softmax_scale, window=window[0])
+    _assert_close("out", out, ref_out, is_f32)
+    _assert_lse(lse, ref_lse, is_f32)
+    dq, dk, dv = hmar.hmar_attn_bwd(tq, tk, tv, out, lse, tdo, wl.side_lens, wl.softmax_scale, window=window[1])
+    rq, rk, rv = orc.attn_bwd(q, k, v, do, wl.side_lens, wl.softmax_scale, window=window[0])
+    _assert_close("dq", dq, rq, is_f32)
+    _assert_close("dk", dk, rk, is_f32)
+    _assert_close("dv", dv, rv, is_f32)
+    _no_device_error()
+
+
+def test_block_causal_full_size_sampled_heads():
+    """The paper's comparison workload (VAR's block-causal mask, App. B.4) on the 512x512 d24 shape."""
+    wl = CONFIGS["512_d24_train"]
+    heads = _sample_heads(wl.B * wl.H, 2)
+    dev, host = training_tensors(wl, heads, with_dout=True)
+    W = hmar.HMAR_WINDOW_CAUSAL
+    out, lse = hmar.hmar_attn_fwd(dev["q"], dev["k"], dev["v"], wl.side_lens, wl.softmax_scale, window=W)
+    idx = torch.as_tensor(heads, device="cuda")
+    ref_out, ref_lse = orc.attn_fwd(host["q"], host["k"], host["v"], wl.side_lens, wl.softmax_scale, window="causal")
+    _assert_close("out", out.view(-1, wl.L, wl.D)[idx], ref_out, False)
+    _assert_lse(lse.view(-1, wl.L)[idx], ref_lse, False)
+    dq, dk, dv = hmar.hmar_attn_bwd(dev["q"], dev["k"], dev["v"], out, lse, dev["dout"], wl.side_lens, wl.softmax_scale, window=W)
+    rq, rk, rv = orc.attn_bwd(host["q"], host["k"], host["v"], host["dout"], wl.side_lens, wl.softmax_scale, window="causal")
+    for nm, g, r in (("dq", dq, rq), ("dk", dk, rk), ("dv", dv, rv)):
+        assert torch.isfinite(g).all()
+        _assert_close(nm, g.view(-1, wl.L, wl.D)[idx], r, False)
+    _no_device_error()
+
+
 def _sample_heads(BH, n=6):
     rng = np.random.default_rng(BH)
     picks = {0, BH - 1} | set(int(x) for x in rng.integers(0, BH, size=n))

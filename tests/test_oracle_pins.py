@@ -88,6 +88,87 @@ def test_block_causal_is_superset_and_denser():
     assert C.sum() > H.sum()
 
 
+# --------------------------------------------------------------------------- the other masks of the family
+
+def test_window_masks_pair_counts_closed_forms():
+    # block-causal: every token of scale k sees start[k+1] tokens; block-diagonal: n_k tokens
+    for sides in (CONFIGS["256_d16_fwd"].side_lens, CONFIGS["512_d24_train"].side_lens, (3, 1, 2)):
+        n = [x * x for x in sides]
+        start = np.concatenate([[0], np.cumsum(n)])
+        assert orc.count_pairs(sides, "causal") == sum(n[k] * start[k + 1] for k in range(len(n)))
+        assert orc.count_pairs(sides, "self") == sum(x * x for x in n)
+    # densities quoted for the paper's shapes: block-causal 61.9 % at L = 680 and 65.2 % at L = 2240
+    assert orc.count_pairs(CONFIGS["256_d16_fwd"].side_lens, "causal") / 680 ** 2 == pytest.approx(0.619, abs=5e-4)
+    assert orc.count_pairs(CONFIGS["512_d24_train"].side_lens, "causal") / 2240 ** 2 == pytest.approx(0.652, abs=5e-4)
+    with pytest.raises(ValueError):
+        orc.window_mask((1, 2), "dense")
+
+
+def test_window_masks_single_scale_all_dense_and_nesting():
+    for w in ("markov", "causal", "self"):
+        assert orc.window_mask((5,), w).all()
+    sides = (2, 3, 1, 4)
+    S, M, C = (orc.window_mask(sides, w) for w in ("self", "markov", "causal"))
+    assert not (S & ~M).any() and not (M & ~C).any() and S.sum() < M.sum() < C.sum()
+    assert (S == S.T).all() and not (C == C.T).all()
+
+
+def test_self_window_is_independent_attention_per_scale():
+    # block-diagonal attention = plain dense attention of every scale on its own (library softmax as the check)
+    rng = np.random.default_rng(11)
+    sides = (2, 3, 1, 4)
+    L = sum(x * x for x in sides)
+    q, k, v = (rng.standard_normal((L, 8)) for _ in range(3))
+    out, lse = orc.attn_fwd(q, k, v, sides, 0.3, window="self")
+    pos = 0
+    for sd in sides:
+        n = sd * sd
+        sl = slice(pos, pos + n)
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(q[sl])[None], torch.from_numpy(k[sl])[None], torch.from_numpy(v[sl])[None], scale=0.3)[0].numpy()
+        np.testing.assert_allclose(out[sl], ref, rtol=1e-12, atol=1e-12)
+        np.testing.assert_allclose(lse[sl], np.log(np.exp(0.3 * q[sl] @ k[sl].T).sum(axis=1)), rtol=1e-12)
+        pos += n
+
+
+def test_causal_window_locality_and_backward():
+    rng = np.random.default_rng(12)
+    sides = (2, 1, 3, 2)
+    n = [x * x for x in sides]
+    start = np.concatenate([[0], np.cumsum(n)])
+    L = int(start[-1])
+    q, k, v, do = (rng.standard_normal((L, 6)) for _ in range(4))
+    out, _ = orc.attn_fwd(q, k, v, sides, 0.4, window="causal")
+    # scale-k rows do not move when a later scale changes, and do move when the first scale changes
+    k2, v2 = k.copy(), v.copy()
+    k2[start[3]:] += 1.0
+    v2[start[3]:] -= 2.0
+    out2, _ = orc.attn_fwd(q, k2, v2, sides, 0.4, window="causal")
+    assert np.array_equal(out[:start[3]], out2[:start[3]]) and not np.allclose(out[start[3]:], out2[start[3]:])
+    v3 = v.copy()
+    v3[0] += 5.0
+    out3, _ = orc.attn_fwd(q, k, v3, sides, 0.4, window="causal")
+    assert not np.allclose(out[start[3]:], out3[start[3]:])          # the last scale still sees token 0
+    outm, _ = orc.attn_fwd(q, k, v3, sides, 0.4)                      # ... which it does not under the Markov mask
+    outm0, _ = orc.attn_fwd(q, k, v, sides, 0.4)
+    assert np.array_equal(outm[start[3]:], outm0[start[3]:])
+    # the last row of a block-causal mask is dense: textbook attention over everything
+    w = np.exp(0.4 * q[-1] @ k.T)
+    np.testing.assert_allclose(out[-1], (w / w.sum()) @ v, rtol=1e-12)
+    # backward by central differences, for both added masks
+    for window in ("causal", "self"):
+        dq, dk, dv = orc.attn_bwd(q, k, v, do, sides, 0.4, window=window)
+        for grad, idx in ((dq, 0), (dk, 1), (dv, 2)):
+            for _ in range(12):
+                i, d = int(rng.integers(L)), int(rng.integers(6))
+                args = [q.copy(), k.copy(), v.copy()]
+                args[idx][i, d] += 1e-6
+                fp = (orc.attn_fwd(*args, sides, 0.4, window=window)[0] * do).sum()
+                args[idx][i, d] -= 2e-6
+                fm = (orc.attn_fwd(*args, sides, 0.4, window=window)[0] * do).sum()
+                assert (fp - fm) / 2e-6 == pytest.approx(grad[i, d], rel=1e-6, abs=1e-8)
+
+
 # --------------------------------------------------------------------------- forward
 
 def _brute_forward(q, k, v, sides, scale):

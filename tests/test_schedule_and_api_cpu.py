@@ -19,14 +19,18 @@ SIDE_LISTS = [
 ]
 
 
+WINDOWS = [("markov", hmar.HMAR_WINDOW_MARKOV), ("causal", hmar.HMAR_WINDOW_CAUSAL), ("self", hmar.HMAR_WINDOW_SELF)]
+
+
+@pytest.mark.parametrize("window", WINDOWS, ids=[w[0] for w in WINDOWS])
 @pytest.mark.parametrize("sides", SIDE_LISTS)
 @pytest.mark.parametrize("direction", [0, 1])
-def test_tiles_cover_exactly_the_live_blocks(sides, direction):
-    M = orc.hmar_mask(sides)
+def test_tiles_cover_exactly_the_live_blocks(sides, direction, window):
+    M = orc.window_mask(sides, window[0])
     if direction == 1:
         M = M.T            # rows = keys, columns = the queries that see them
     L = M.shape[0]
-    tiles = hmar.hmar_schedule_tiles(sides, direction)
+    tiles = hmar.hmar_schedule_tiles(sides, direction, window=window[1])
     seen = np.zeros(L, dtype=int)
     for t in tiles:
         r0, rc = t["row_begin"], t["row_count"]
