@@ -176,6 +176,32 @@ def time_scale_steps(hmar, wl_inf, dev, reps=5):
     return out
 
 
+def time_training_shape(hmar, wl_x, dev, window, reps=3):
+    """ms of forward and of backward on another training shape / mask of the family (context legs)."""
+    import torch
+    from workloads.device import bulk_normal
+    B, H, L, D = wl_x.B, wl_x.H, wl_x.L, wl_x.D
+    q, k, v, do = (bulk_normal(wl_x.seed, i, B, H, L, D, torch.bfloat16, dev) for i in range(4))
+    out = torch.empty_like(q)
+    lse = torch.empty((B, H, L), dtype=torch.float32, device=dev)
+    dq, dk, dv = (torch.empty_like(q) for _ in range(3))
+    ws = torch.empty(hmar.hmar_attn_bwd_workspace_bytes(B, H, D, wl_x.side_lens), dtype=torch.uint8, device=dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    f_ms = b_ms = 0.0
+    for it in range(reps + 1):
+        ev[0].record()
+        hmar.hmar_attn_fwd(q, k, v, wl_x.side_lens, wl_x.softmax_scale, out=out, lse=lse, window=window)
+        ev[1].record()
+        hmar.hmar_attn_bwd(q, k, v, out, lse, do, wl_x.side_lens, wl_x.softmax_scale, dq=dq, dk=dk, dv=dv,
+                           workspace=ws, window=window)
+        ev[2].record()
+        torch.cuda.synchronize()
+        if it:
+            f_ms += ev[0].elapsed_time(ev[1]) / reps
+            b_ms += ev[1].elapsed_time(ev[2]) / reps
+    return f_ms, b_ms
+
+
 def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -279,6 +305,20 @@ def run_ours(args, wl):
             ms = time_scale_steps(hmar, CONFIGS["512_d24_infer"], dev)
             extras["scale_step_ms"] = {"workload": "512_d24_infer, B=64 H=24, one sub-step per call", "per_scale": ms,
                                        "sweep_4_sub_steps": round(4 * sum(ms), 4)}
+            torch.cuda.empty_cache()
+            # VAR's block-causal mask on the same shape and kernels: the workload the paper's speedups are against
+            cf, cb = time_training_shape(hmar, wl, dev, hmar.HMAR_WINDOW_CAUSAL)
+            extras["block_causal_same_kernels"] = {"fwd_ms": round(cf, 4), "bwd_ms": round(cb, 4),
+                                                   "markov_speedup_fwd": round(cf / fwd_ms, 3),
+                                                   "markov_speedup_bwd": round(cb / bwd_ms, 3)}
+            torch.cuda.empty_cache()
+            # 1024 x 1024 (synthetic 14-scale schedule ending at 64 x 64, L = 9451), Markov mask
+            wl_big = CONFIGS["1024_d24_train"]
+            bf, bb = time_training_shape(hmar, wl_big, dev, hmar.HMAR_WINDOW_MARKOV, reps=2)
+            fl_f, fl_b = useful_flops(wl_big)
+            extras["1024_d24_train"] = {"L": wl_big.L, "fwd_ms": round(bf, 4), "bwd_ms": round(bb, 4),
+                                        "useful_tflops": round((fl_f + fl_b) / ((bf + bb) * 1e-3) / 1e12, 1),
+                                        "schedule": "synthetic: " + str(list(wl_big.side_lens))}
             torch.cuda.empty_cache()
     args.extras = extras
 

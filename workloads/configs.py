@@ -11,6 +11,9 @@ from typing import Tuple
 SIDES_TINY = (1, 2, 3, 4)
 SIDES_256 = (1, 2, 3, 4, 5, 6, 8, 10, 13, 16)
 SIDES_512 = (1, 2, 3, 4, 6, 9, 13, 18, 24, 32)
+# 1024x1024: the paper benchmarks this resolution (App. B.4) but prints no schedule for it; this one is
+# synthetic (the 512 schedule's growth continued to a 64 x 64 last scale, 14 scales).
+SIDES_1024 = (1, 2, 3, 4, 5, 7, 9, 12, 16, 21, 27, 36, 48, 64)
 
 BASE_SEED = 20250604 * 10
 
@@ -42,6 +45,7 @@ CONFIGS = {
     "256_d30_train": Workload("256_d30_train", 3, 32, 30, 64, SIDES_256, 0.125, ("fwd", "bwd")),
     "512_d24_train": Workload("512_d24_train", 4, 16, 24, 64, SIDES_512, 0.125, ("fwd", "bwd")),
     "512_d24_infer": Workload("512_d24_infer", 5, 64, 24, 64, SIDES_512, 0.125, ("scale_step",), 4),
+    "1024_d24_train": Workload("1024_d24_train", 6, 16, 24, 64, SIDES_1024, 0.125, ("fwd", "bwd")),
 }
 
 
