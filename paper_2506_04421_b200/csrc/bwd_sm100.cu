@@ -54,9 +54,9 @@ constexpr int NUM_COMPUTE_THREADS = 256;
 constexpr int DRAIN_WARP0 = 8, PRODUCER_WARP = 12, MMA_WARP = 13, AUX_WARP = 14;
 constexpr int NUM_THREADS = 512;
 #ifndef X_RC
-#define X_RC 160
-#define X_RD 72
-#define X_RM 120
+#define X_RC 152
+#define X_RD 96
+#define X_RM 112
 #endif
 constexpr int REGS_COMPUTE = X_RC, REGS_DRAIN = X_RD, REGS_MISC = X_RM;
 static_assert(2 * REGS_COMPUTE + REGS_DRAIN + REGS_MISC == 4 * 128, "register budget of the block");
@@ -64,15 +64,15 @@ constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t COL_ST = 0, COL_DPT = 128, COL_DK = 256, COL_DV = 320, COL_DQ = 384, COL_K = 448, COL_V = 480;
 
 struct __align__(1024) SharedStorage {
-    uint8_t k[TILE_BYTES];
-    uint8_t v[TILE_BYTES];
+    uint8_t k[2][TILE_BYTES];               // K of the current item and of the next one (B operand of dQ)
     uint8_t q[NSTAGE][TILE_BYTES];
     uint8_t dout[NSTAGE][TILE_BYTES];
     uint8_t ds[2][2][TILE_BYTES];           // dS^T, double buffered: [step parity][64-query half][key row][64 queries], 128B swizzle
     uint8_t dq_stage[TILE_BYTES];           // per drain warp: 32 query rows x 32 fp32 columns of dQ_i on their way to the accumulator, 128B swizzle
     float lse2[AUX_STAGES][BQ];             // lse * log2(e); +inf for query rows outside the range
     float delta[AUX_STAGES][BQ];
-    uint64_t kv_full, kv_tmem;
+    uint64_t k_full[2], k_free[2];          // [item parity]: K tile in shared memory / no longer read
+    uint64_t kv_tmem, kv_free;              // K, V rows in TMEM / no longer read
     uint64_t qdo_full[NSTAGE], q_empty[NSTAGE], aux_full[AUX_STAGES], aux_empty[AUX_STAGES];
     uint64_t s_full[2], p_full[2];            // [half of the step]
     uint64_t dq_full, dq_empty, acc_full, acc_empty;
@@ -130,8 +130,12 @@ __device__ __forceinline__ void load_swizzled_row(const uint8_t* tile, int r, ui
 // (the 32 packed columns start at the half's first column, which this warp has already read for these
 // rows), and dS^T also goes to shared memory, 4 bytes per pair (a warp's store covers 16 bytes of 8 rows,
 // 128-byte swizzle on the key row: no bank conflicts).
-// MASKED: row i of this thread's four rows sees only columns [c_lo[i], c_hi[i]) of the step.
-template <bool MASKED>
+// MODE 2: row i of this thread's four rows sees only columns [c_lo[i], c_hi[i]) of the step.
+// MODE 1: every row either sees all columns or is past the end of the key tile (c_hi[i] <= 0).  Such a row
+// holds another tile's keys; its P^T and dS^T only reach rows of dV and dK that are never written, but in
+// dQ = dS K it would be summed over, so the copy of dS in shared memory gets zeros there.
+// MODE 0: all rows see all columns.
+template <int MODE>
 __device__ __forceinline__ void softmax_grad_half(uint32_t lane_base, int cbase, const float* lse2, const float* delta,
                                                   float sl2, const int (&c_lo)[4], const int (&c_hi)[4], uint8_t* ds_tile,
                                                   int quarter, int lane) {
@@ -158,7 +162,7 @@ __device__ __forceinline__ void softmax_grad_half(uint32_t lane_base, int cbase,
             for (int rs = 0; rs < 2; ++rs) {
                 float p0 = ex2(fmaf(__uint_as_float(s_buf[4 * k + 2 * rs]), sl2, -ls[k].x));
                 float p1 = ex2(fmaf(__uint_as_float(s_buf[4 * k + 2 * rs + 1]), sl2, -ls[k].y));
-                if (MASKED) {
+                if (MODE == 2) {
                     const int c = cbase + 8 * k + 2 * tq, i = hl * 2 + rs;
                     p0 = (c >= c_lo[i] && c < c_hi[i]) ? p0 : 0.f;
                     p1 = (c + 1 >= c_lo[i] && c + 1 < c_hi[i]) ? p1 : 0.f;
@@ -168,7 +172,8 @@ __device__ __forceinline__ void softmax_grad_half(uint32_t lane_base, int cbase,
                 p_pack[2 * k + rs] = pack_bf16(p0, p1);
                 ds_pack[2 * k + rs] = pack_bf16(d0, d1);
                 // 8-row groups are 1024 bytes apart; 16-byte piece k of a row sits at position k ^ (row & 7)
-                *reinterpret_cast<uint32_t*>(ds_row + rs * 1024 + ((k ^ tr) << 4)) = ds_pack[2 * k + rs];
+                *reinterpret_cast<uint32_t*>(ds_row + rs * 1024 + ((k ^ tr) << 4)) =
+                    (MODE == 1 && c_hi[hl * 2 + rs] <= 0) ? 0u : ds_pack[2 * k + rs];
             }
         }
         tmem_st_16x128b_x8(taddr + COL_ST + cbase, p_pack);
@@ -207,8 +212,12 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 
     if (threadIdx.x == 0) {
         sm.abort_flag = 0;
-        mbar_init(&sm.kv_full, 1);
-        mbar_init(&sm.kv_tmem, NUM_COMPUTE_THREADS);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sm.k_full[b], 1);
+            mbar_init(&sm.k_free[b], 1);
+        }
+        mbar_init(&sm.kv_tmem, 128);
+        mbar_init(&sm.kv_free, 1);
         for (int s = 0; s < NSTAGE; ++s) {
             mbar_init(&sm.qdo_full[s], 1);
             mbar_init(&sm.q_empty[s], 1);
@@ -224,7 +233,7 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         mbar_init(&sm.dq_full, 1);
         mbar_init(&sm.dq_empty, 128);
         mbar_init(&sm.acc_full, 1);
-        mbar_init(&sm.acc_empty, NUM_COMPUTE_THREADS);
+        mbar_init(&sm.acc_empty, 128);
         fence_mbar_init();
         const long long total = (long long)args.n_heads * args.head_cost;
         sm.item_begin = first_item_at_cost(args, total * blockIdx.x / gridDim.x);
@@ -273,15 +282,17 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 const int bh = g / n_work;
                 const BwdWork w = get_work(g);
                 const int n_steps = steps_of(w);
-                if (g > item_begin) {
-                    // K in shared memory is read by the dQ products until the previous item is complete
-                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.acc_full, (g - item_begin - 1) & 1, abort_flag));
+                const int item = g - item_begin;
+                if (item >= 2) {
+                    // the buffer held K of the item before the previous one, read by its dQ products
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.k_free[item & 1], ((item >> 1) & 1) ^ 1, abort_flag));
                     if (!ok) { if (lane == 0) report_timeout(args.status, 0x1000); break; }
                 }
                 if (leader) {
-                    mbar_arrive_expect_tx(&sm.kv_full, 2 * TILE_BYTES);
-                    tma_load_3d(sm.k, &map_k, &sm.kv_full, 0, w.row_begin, bh);
-                    tma_load_3d(sm.v, &map_v, &sm.kv_full, 0, w.row_begin, bh);
+                    mbar_arrive_expect_tx(&sm.k_full[item & 1], TILE_BYTES);
+                    tma_load_3d(sm.k[item & 1], &map_k, &sm.k_full[item & 1], 0, w.row_begin, bh);
+                    // the V rows are read by the drain warps a few steps from now: bring them into L2
+                    tma_prefetch_3d(&map_v, 0, w.row_begin, bh);
                 }
                 __syncwarp();
                 for (int i = 0; i < n_steps; ++i, ++gs) {
@@ -350,7 +361,7 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             //   Y_i = dV,dK of half 1 of step i, then S^T,dP^T of half 1 of step i+1, then dQ_i
             // each preceded by one look at the barriers it depends on (two at a time, both usually complete).
             const bool leader = elect_one();
-            const uint64_t k_mn = smem_desc_sw128(smem_u32(sm.k), 1024);        // K as MN-major B of dQ
+            const uint64_t k_mn0 = smem_desc_sw128(smem_u32(sm.k[0]), 1024);    // K as MN-major B of dQ
             // the ring slots and the dS buffers are 16 KB apart: descriptor of slot s = base + s * 1024
             const uint64_t q_kd0 = smem_desc_sw128(smem_u32(sm.q[0]), 16), do_kd0 = smem_desc_sw128(smem_u32(sm.dout[0]), 16);
             const uint64_t q_mn0 = smem_desc_sw128(smem_u32(sm.q[0]), 1024), do_mn0 = smem_desc_sw128(smem_u32(sm.dout[0]), 1024);
@@ -396,35 +407,58 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         mma_ts(tmem + COL_DK, tmem + COL_DPT + h * HQ + ks * 8, qd + ks * 128, idesc_acc, !first || (ks > 0));
             };
 
+            auto wait1 = [&](uint64_t* a, uint32_t pa, int code) -> bool {
+                if (__all_sync(0xffffffffu, mbar_wait(a, pa, abort_flag))) return true;
+                if (lane == 0) report_timeout(args.status, code);
+                return false;
+            };
+            // The steps of all items form one sequence: while the compute warpgroups work on a step, the
+            // tensor core gets the next step's S^T, dP^T even when that step belongs to the next item (whose
+            // K, V rows the drain warps have put into TMEM by then).
+            if (item_begin < item_end) {
+                const BwdWork w0 = get_work(item_begin);
+                ok = wait2(&sm.kv_tmem, 0, &sm.qdo_full[0], 0, true, 0x1200);
+                if (ok) {
+                    tc_fence_after();
+                    if (leader) {
+                        scores(0, half_cols(w0, 0, 0), 0);
+                        const int n1 = half_cols(w0, 0, 1);
+                        if (n1 > 0) scores(1, n1, 0);
+                        if (steps_of(w0) == 1 && item_begin + 1 < item_end) tc_commit(&sm.kv_free);
+                    }
+                    __syncwarp();
+                }
+            }
             for (int g = item_begin; g < item_end && ok; ++g) {
                 const BwdWork w = get_work(g);
                 const int n_steps = steps_of(w);
                 const int item = g - item_begin;
-
-                // K and V of this item are in TMEM (the compute warps copy them after the previous item's end)
-                ok = wait2(&sm.kv_tmem, item & 1, &sm.qdo_full[gs % NSTAGE], (gs / NSTAGE) & 1, true, 0x1200);
-                if (!ok) break;
-                tc_fence_after();
-                if (leader) {
-                    scores(0, half_cols(w, 0, 0), gs % NSTAGE);
-                    const int n1 = half_cols(w, 0, 1);
-                    if (n1 > 0) scores(1, n1, gs % NSTAGE);
-                }
-                __syncwarp();
-                // dK and dV of the previous item must have been read out before they are overwritten
-                if (item > 0) {
-                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.acc_empty, (item - 1) & 1, abort_flag));
-                    if (!ok) { if (lane == 0) report_timeout(args.status, 0x1B00); break; }
-                }
+                const bool next_item = g + 1 < item_end;
+                const BwdWork wn = next_item ? get_work(g + 1) : w;
+                const int n_steps_next = steps_of(wn);
+                const uint64_t k_mn = k_mn0 + (item & 1) * 1024;
                 for (int i = 0; i < n_steps && ok; ++i, ++gs) {
                     const int slot = gs % NSTAGE, slot_next = (gs + 1) % NSTAGE;
-                    const bool more = i + 1 < n_steps;
+                    const bool more = i + 1 < n_steps;          // the item has another step
+                    const bool cross = !more && next_item;      // the next step is the next item's first
+                    const bool any_next = more || cross;
                     const int n0 = half_cols(w, i, 0), n1 = half_cols(w, i, 1);
-                    const int m0 = more ? half_cols(w, i + 1, 0) : 0, m1 = more ? half_cols(w, i + 1, 1) : 0;
+                    const int m0 = more ? half_cols(w, i + 1, 0) : cross ? half_cols(wn, 0, 0) : 0;
+                    const int m1 = more ? half_cols(w, i + 1, 1) : cross ? half_cols(wn, 0, 1) : 0;
+                    // the next step is the last one that reads its item's K, V rows in TMEM, and another item follows
+                    const bool frees_kv = more ? (i + 2 == n_steps && next_item) : (cross && n_steps_next == 1 && g + 2 < item_end);
                     // ---- burst X: needs P^T, dS^T of half 0 and the next step's Q / dO tile
-                    ok = wait2(&sm.p_full[0], ng[0] & 1, &sm.qdo_full[slot_next], ((gs + 1) / NSTAGE) & 1, more, 0x1400 + i);
+                    ok = wait2(&sm.p_full[0], ng[0] & 1, &sm.qdo_full[slot_next], ((gs + 1) / NSTAGE) & 1, any_next, 0x1400 + i);
                     if (!ok) break;
                     ++ng[0];
+                    if (cross) {                                // K, V of the next item in TMEM
+                        ok = wait1(&sm.kv_tmem, (item + 1) & 1, 0x1200);
+                        if (!ok) break;
+                    }
+                    if (i == 0 && item > 0) {                   // dK, dV of the previous item read out
+                        ok = wait1(&sm.acc_empty, (item - 1) & 1, 0x1B00);
+                        if (!ok) break;
+                    }
                     tc_fence_after();
                     if (leader) {
                         grads(0, n0, slot, i == 0);
@@ -440,13 +474,19 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         ok = wait2(&sm.dq_empty, (gs - 1) & 1, nullptr, 0, false, 0x1800 + i);
                     }
                     if (!ok) break;
+                    if (i == 0) {                               // K of this item in shared memory (B operand of dQ)
+                        ok = wait1(&sm.k_full[item & 1], (item >> 1) & 1, 0x1C00);
+                        if (!ok) break;
+                    }
                     tc_fence_after();
                     if (leader) {
                         if (n1 > 0) grads(1, n1, slot, false);
                         tc_commit(&sm.q_empty[slot]);           // Q_i, dO_i are not read again
+                        if (!more) tc_commit(&sm.acc_full);     // dK, dV of the item are complete
                         // the next scores of half 1 go first: the compute warpgroup is waiting for them, dQ_i
                         // is not needed before the drain warps get to it
                         if (m1 > 0) scores(1, m1, slot_next);
+                        if (frees_kv) tc_commit(&sm.kv_free);
                         // dQ_i = dS K over both halves: A = dS (queries x keys) read as an MN-major operand.  When
                         // the step has no second half its rows are stale data and are never drained.
                         const uint64_t dsd = ds_mn0 + (gs & 1) * 2048;
@@ -454,7 +494,7 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         for (int ks = 0; ks < BKV / 16; ++ks)
                             mma_ss(tmem + COL_DQ, dsd + ks * 128, k_mn + ks * 128, idesc_dq, ks > 0);
                         tc_commit(&sm.dq_full);
-                        if (!more) tc_commit(&sm.acc_full);
+                        if (!more) tc_commit(&sm.k_free[item & 1]);
                     }
                     __syncwarp();
                 }
@@ -477,11 +517,87 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         uint32_t buf[32];
         bool ok = true;
         int gs = 0;
+        auto wait1 = [&](uint64_t* a, uint32_t pa, int code) -> bool {
+            if (__all_sync(0xffffffffu, mbar_wait(a, pa, abort_flag))) return true;
+            if (lane == 0) report_timeout(args.status, code);
+            return false;
+        };
+        // K and V rows of item gc (the block's item number `item`) to TMEM, one key row per thread: the A
+        // operands of S^T = K Q^T and dP^T = V dO^T.  The V row comes straight from global memory and waits
+        // in registers until the previous item's last scores have been computed; the K row is read from the
+        // tile that the copy engine has put into shared memory for the dQ products.  Rows past the end of
+        // the sequence are zeros.
+        auto copy_kv = [&](int gc, int item, bool wait_free) -> bool {
+            const BwdWork wc = get_work(gc);
+            const int row = wc.row_begin + r;
+            const uint4* vsrc = reinterpret_cast<const uint4*>(args.v + ((size_t)(gc / n_work) * L + row) * D);
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const uint4 val = row < L ? __ldg(vsrc + c) : make_uint4(0u, 0u, 0u, 0u);
+                buf[4 * c] = val.x; buf[4 * c + 1] = val.y; buf[4 * c + 2] = val.z; buf[4 * c + 3] = val.w;
+            }
+            if (wait_free) {
+                if (!wait1(&sm.kv_free, (item - 1) & 1, 0x1900)) return false;
+                tc_fence_after();
+            }
+            tmem_st32(lane_base + COL_V, buf);
+            if (!wait1(&sm.k_full[item & 1], (item >> 1) & 1, 0x1980)) return false;
+            load_swizzled_row(sm.k[item & 1], r, buf);
+            tmem_st32(lane_base + COL_K, buf);
+            tmem_st_wait();
+            tc_fence_before();
+            mbar_arrive(&sm.kv_tmem);
+            return true;
+        };
+        if (item_begin < item_end) {
+            ok = copy_kv(item_begin, 0, false);
+            if (ok && steps_of(get_work(item_begin)) == 1 && item_begin + 1 < item_end) ok = copy_kv(item_begin + 1, 1, true);
+        }
         for (int g = item_begin; g < item_end && ok; ++g) {
             const int bh = g / n_work;
             const BwdWork w = get_work(g);
             const int n_steps = steps_of(w);
+            const int item = g - item_begin;
+            const bool next_item = g + 1 < item_end;
+            const int n_steps_next = next_item ? steps_of(get_work(g + 1)) : 0;
             for (int i = 0; i < n_steps; ++i, ++gs) {
+                const bool more = i + 1 < n_steps;
+                // the next step is the last one of its item and another item follows: that item's K, V rows
+                // go to TMEM as soon as the next step's scores are complete
+                if (more ? (i + 2 == n_steps && next_item) : (next_item && n_steps_next == 1 && g + 2 < item_end)) {
+                    const int gc = more ? g + 1 : g + 2;
+                    ok = copy_kv(gc, gc - item_begin, true);
+                    if (!ok) break;
+                }
+                if (!more) {
+                    // ---- end of the item: dK and dV, one key row per thread, scaled and rounded to bf16
+                    ok = wait1(&sm.acc_full, item & 1, 0x1A00);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int part = 0; part < 4; ++part) {
+                        tmem_ld32(lane_base + (part < 2 ? COL_DK : COL_DV) + (part & 1) * 32, buf);
+                        tmem_ld_wait();
+                        if (part == 3) {
+                            tc_fence_before();
+                            mbar_arrive(&sm.acc_empty);         // the next item's products may overwrite dK / dV
+                        }
+                        if (r < w.row_count) {
+                            const float mul = part < 2 ? args.softmax_scale : 1.f;
+                            __nv_bfloat16* base = part < 2 ? args.dk : args.dv;
+                            uint4* dst = reinterpret_cast<uint4*>(base + ((size_t)bh * L + w.row_begin + r) * D + (part & 1) * 32);
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) {
+                                uint4 o;
+                                o.x = pack_bf16(__uint_as_float(buf[8 * t + 0]) * mul, __uint_as_float(buf[8 * t + 1]) * mul);
+                                o.y = pack_bf16(__uint_as_float(buf[8 * t + 2]) * mul, __uint_as_float(buf[8 * t + 3]) * mul);
+                                o.z = pack_bf16(__uint_as_float(buf[8 * t + 4]) * mul, __uint_as_float(buf[8 * t + 5]) * mul);
+                                o.w = pack_bf16(__uint_as_float(buf[8 * t + 6]) * mul, __uint_as_float(buf[8 * t + 7]) * mul);
+                                dst[t] = o;
+                            }
+                        }
+                    }
+                }
                 if (!__all_sync(0xffffffffu, mbar_wait(&sm.dq_full, gs & 1, abort_flag))) {
                     if (lane == 0) report_timeout(args.status, 0x1600 + i);
                     ok = false;
@@ -522,22 +638,18 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         reg_inc<REGS_COMPUTE>();
         const int quarter = warp & 3;
         const int h = warp >> 2;                            // the half of every step this warpgroup owns
-        const int j = quarter * 32 + lane;                  // key row inside the tile
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
         const float sl2 = args.scale_log2;
-        uint32_t s_buf[32], dp_buf[32];                     // K / V row on its way to TMEM; dK / dV row at the end of an item
         bool ok = true;
         int gs = 0;                                         // steps seen so far (aux ring, dS buffer parity)
         int nsh = 0;                                        // non-empty halves of this warpgroup seen so far
 
         for (int g = item_begin; g < item_end && ok; ++g) {
-            const int bh = g / n_work;
             const BwdWork w = get_work(g);
             const int n_steps = steps_of(w);
-            const int item = g - item_begin;
-            const bool row_ok = j < w.row_count;            // this thread's row in the 32x32b layout (K / V copy, dK / dV)
             // the four key rows this thread works on in the softmax-gradient layout, and the queries that may see them
             const bool tile_masked = (!w.uniform) || (w.row_count < BKV);
+            const bool rows_only = w.uniform != 0;          // only rows past the end of the tile are hidden
             int qlo[4], qhi[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -552,15 +664,6 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     }
                 }
             }
-
-            // ---- K (warpgroup 0) / V (warpgroup 1) row to TMEM: A operands of S^T = K Q^T and dP^T = V dO^T
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.kv_full, item & 1, abort_flag));
-            if (!ok) { if (lane == 0) report_timeout(args.status, 0x1900); break; }
-            load_swizzled_row(h == 0 ? sm.k : sm.v, j, s_buf);
-            tmem_st32(lane_base + (h == 0 ? COL_K : COL_V), s_buf);
-            tmem_st_wait();
-            tc_fence_before();
-            mbar_arrive(&sm.kv_tmem);
 
             for (int i = 0; i < n_steps && ok; ++i, ++gs) {
                 const int q0 = w.q_begin + i * BQ;
@@ -585,11 +688,15 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                             c_lo[r4] = max(qlo[r4] - q0, 0);
                             c_hi[r4] = min(qhi[r4] - q0, n_valid);
                         }
-                        softmax_grad_half<true>(lane_base, cbase, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi,
-                                                sm.ds[gs & 1][h], quarter, lane);
+                        if (rows_only)
+                            softmax_grad_half<1>(lane_base, cbase, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi,
+                                                 sm.ds[gs & 1][h], quarter, lane);
+                        else
+                            softmax_grad_half<2>(lane_base, cbase, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi,
+                                                 sm.ds[gs & 1][h], quarter, lane);
                     } else {
                         const int none[4] = {0, 0, 0, 0};
-                        softmax_grad_half<false>(lane_base, cbase, sm.lse2[aslot], sm.delta[aslot], sl2, none, none,
+                        softmax_grad_half<0>(lane_base, cbase, sm.lse2[aslot], sm.delta[aslot], sl2, none, none,
                                                  sm.ds[gs & 1][h], quarter, lane);
                     }
                     tmem_st_wait();
@@ -598,40 +705,6 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     mbar_arrive(&sm.p_full[h]);
                 }
                 mbar_arrive(&sm.aux_empty[aslot]);      // this thread is done with the step's lse / delta
-            }
-            if (!ok) break;
-
-            // ---- end of the item: dK (warpgroup 0) and dV (warpgroup 1), one key row per thread
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.acc_full, item & 1, abort_flag));
-            if (!ok) { if (lane == 0) report_timeout(args.status, 0x1A00); break; }
-            tc_fence_after();
-            tmem_ld32(lane_base + (h == 0 ? COL_DK : COL_DV), s_buf);
-            tmem_ld32(lane_base + (h == 0 ? COL_DK : COL_DV) + 32, dp_buf);
-            tmem_ld_wait();
-            tc_fence_before();
-            mbar_arrive(&sm.acc_empty);                 // the next item's products may overwrite dK / dV
-            if (row_ok) {
-                const float mul = h == 0 ? args.softmax_scale : 1.f;
-                __nv_bfloat16* base = h == 0 ? args.dk : args.dv;
-                uint4* dst = reinterpret_cast<uint4*>(base + ((size_t)bh * L + w.row_begin + j) * D);
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    uint4 o;
-                    o.x = pack_bf16(__uint_as_float(s_buf[8 * t + 0]) * mul, __uint_as_float(s_buf[8 * t + 1]) * mul);
-                    o.y = pack_bf16(__uint_as_float(s_buf[8 * t + 2]) * mul, __uint_as_float(s_buf[8 * t + 3]) * mul);
-                    o.z = pack_bf16(__uint_as_float(s_buf[8 * t + 4]) * mul, __uint_as_float(s_buf[8 * t + 5]) * mul);
-                    o.w = pack_bf16(__uint_as_float(s_buf[8 * t + 6]) * mul, __uint_as_float(s_buf[8 * t + 7]) * mul);
-                    dst[t] = o;
-                }
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    uint4 o;
-                    o.x = pack_bf16(__uint_as_float(dp_buf[8 * t + 0]) * mul, __uint_as_float(dp_buf[8 * t + 1]) * mul);
-                    o.y = pack_bf16(__uint_as_float(dp_buf[8 * t + 2]) * mul, __uint_as_float(dp_buf[8 * t + 3]) * mul);
-                    o.z = pack_bf16(__uint_as_float(dp_buf[8 * t + 4]) * mul, __uint_as_float(dp_buf[8 * t + 5]) * mul);
-                    o.w = pack_bf16(__uint_as_float(dp_buf[8 * t + 6]) * mul, __uint_as_float(dp_buf[8 * t + 7]) * mul);
-                    dst[4 + t] = o;
-                }
             }
         }
     }

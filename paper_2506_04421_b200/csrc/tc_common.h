@@ -61,6 +61,8 @@ struct BwdArgs {
     const float* delta;      // [BH, L] rowsum(dO o O) (read by the main kernel)
     float* delta_w;          // same buffer, written by the preprocess kernel
     float* dq_acc;           // [BH, L, 64] fp32 accumulator
+    const __nv_bfloat16* k;  // [BH, L, 64] (read directly for the rows that go to TMEM)
+    const __nv_bfloat16* v;
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     int* status;

@@ -226,6 +226,8 @@ int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const f
     a.delta = delta;
     a.delta_w = delta;
     a.dq_acc = dq_acc;
+    a.k = k;
+    a.v = v;
     a.dk = dk;
     a.dv = dv;
     a.status = status;
