@@ -120,51 +120,47 @@ __device__ __forceinline__ void load_swizzled_row(const uint8_t* tile, int r, ui
     }
 }
 
-// 32 query columns (starting at column c0 of the step) for the 32 key rows of one warp:
+// The 64 query columns of one half step for the 32 key rows of one warp:
 // P^T = 2^(S^T * scale * log2e - lse * log2e) and dS^T = P^T o (dP^T - delta) in fp32.
 // S^T and dP^T are read 16 key rows at a time in the layout in which a thread holds, of two rows, the
-// column pairs 8k + 2(t % 4) + {0, 1}: a thread then needs lse and delta of 8 columns only (four 8-byte
-// loads each, one shared-memory wavefront per load; one key row per thread would need every column as a
-// broadcast load, which was the largest share of the shared-memory traffic of the LSU).  A column pair
+// column pairs 8k + 2(t % 4) + {0, 1}: a thread then needs lse and delta of 16 columns only (eight 8-byte
+// loads each, one shared-memory wavefront per load; one key row per thread would need all 64 columns as
+// broadcast loads, which were the largest share of the shared-memory traffic of the LSU).  A column pair
 // packs into one bf16x2: P^T goes back to TMEM over S^T and dS^T over dP^T with the matching store layout
-// (the 16 packed columns start at c0, which this warp has already read for these rows), and dS^T also goes
-// to shared memory, 4 bytes per pair (a warp's store covers 16 bytes of 8 rows, 128-byte swizzle on the key
-// row: no bank conflicts); in the 64-query buffer ds_tile the columns start at 16-byte piece `piece0` of a row.
-// The arithmetic works on pairs of columns with packed fp32 instructions (half as many to issue and to fetch).
+// (the 32 packed columns start at the half's first column, which this warp has already read for these
+// rows), and dS^T also goes to shared memory, 4 bytes per pair (a warp's store covers 16 bytes of 8 rows,
+// 128-byte swizzle on the key row: no bank conflicts).
 // MODE 2: row i of this thread's four rows sees only columns [c_lo[i], c_hi[i]) of the step.
 // MODE 1: every row either sees all columns or is past the end of the key tile (c_hi[i] <= 0).  Such a row
 // holds another tile's keys; its P^T and dS^T only reach rows of dV and dK that are never written, but in
 // dQ = dS K it would be summed over, so the copy of dS in shared memory gets zeros there.
 // MODE 0: all rows see all columns.
 template <int MODE>
-__device__ __forceinline__ void softmax_grad_cols(uint32_t lane_base, int c0, int piece0, const float* neg_lse2,
-                                                  const float* neg_delta, float sl2, const int (&c_lo)[4],
-                                                  const int (&c_hi)[4], uint8_t* ds_tile, int quarter, int lane) {
+__device__ __forceinline__ void softmax_grad_half(uint32_t lane_base, int cbase, const float* neg_lse2, const float* neg_delta,
+                                                  float sl2, const int (&c_lo)[4], const int (&c_hi)[4], uint8_t* ds_tile,
+                                                  int quarter, int lane) {
     const int tq = lane & 3, tr = lane >> 2;
-    uint64_t nls[4], nde[4];                // -lse * log2(e) and -delta of this thread's column pairs
+    // -lse * log2(e) and -delta of this thread's column pairs; the arithmetic works on pairs of columns
+    // with packed fp32 instructions (half as many instructions to issue and to fetch)
+    uint64_t nls[8], nde[8];
 #pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        nls[k] = *reinterpret_cast<const uint64_t*>(neg_lse2 + c0 + 8 * k + 2 * tq);
-        nde[k] = *reinterpret_cast<const uint64_t*>(neg_delta + c0 + 8 * k + 2 * tq);
+    for (int k = 0; k < 8; ++k) {
+        nls[k] = *reinterpret_cast<const uint64_t*>(neg_lse2 + cbase + 8 * k + 2 * tq);
+        nde[k] = *reinterpret_cast<const uint64_t*>(neg_delta + cbase + 8 * k + 2 * tq);
     }
     const uint64_t sl2_2 = f32x2(sl2, sl2);
-    // both 16-lane halves of the warp's rows are requested before the first is worked on
-    uint32_t s_a[16], d_a[16], s_b[16], d_b[16];
-    const uint32_t ta = lane_base, tb = lane_base + (16u << 16);
-    tmem_ld_16x256b_x4(ta + COL_ST + c0, s_a);
-    tmem_ld_16x256b_x4(ta + COL_DPT + c0, d_a);
-    tmem_ld_16x256b_x4(tb + COL_ST + c0, s_b);
-    tmem_ld_16x256b_x4(tb + COL_DPT + c0, d_b);
-    tmem_ld_wait();
 #pragma unroll
     for (int hl = 0; hl < 2; ++hl) {                    // lanes 0-15, then 16-31 of the warp's quarter
-        uint32_t (&s_buf)[16] = hl == 0 ? s_a : s_b;
-        uint32_t (&dp_buf)[16] = hl == 0 ? d_a : d_b;
-        uint32_t p_pack[8], ds_pack[8];
+        const uint32_t taddr = lane_base + ((uint32_t)(hl * 16) << 16);
+        uint32_t s_buf[32], dp_buf[32];
+        tmem_ld_16x256b_x8(taddr + COL_ST + cbase, s_buf);
+        tmem_ld_16x256b_x8(taddr + COL_DPT + cbase, dp_buf);
+        tmem_ld_wait();
+        uint32_t p_pack[16], ds_pack[16];
         // key rows of this thread: quarter * 32 + hl * 16 + tr (+ 8); both have (row & 7) == tr
         uint8_t* ds_row = ds_tile + (quarter * 4 + hl * 2) * 1024 + tr * 128 + tq * 4;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {
+        for (int k = 0; k < 8; ++k) {
 #pragma unroll
             for (int rs = 0; rs < 2; ++rs) {
                 float x0, x1;
@@ -172,7 +168,7 @@ __device__ __forceinline__ void softmax_grad_cols(uint32_t lane_base, int c0, in
                                   sl2_2, nls[k]), x0, x1);
                 float p0 = ex2(x0), p1 = ex2(x1);
                 if (MODE == 2) {
-                    const int c = c0 + 8 * k + 2 * tq, i = hl * 2 + rs;
+                    const int c = cbase + 8 * k + 2 * tq, i = hl * 2 + rs;
                     p0 = (c >= c_lo[i] && c < c_hi[i]) ? p0 : 0.f;
                     p1 = (c + 1 >= c_lo[i] && c + 1 < c_hi[i]) ? p1 : 0.f;
                 }
@@ -182,14 +178,13 @@ __device__ __forceinline__ void softmax_grad_cols(uint32_t lane_base, int c0, in
                                         nde[k])), d0, d1);
                 p_pack[2 * k + rs] = pack_bf16(p0, p1);
                 ds_pack[2 * k + rs] = pack_bf16(d0, d1);
-                // 8-row groups are 1024 bytes apart; 16-byte piece p of a row sits at position p ^ (row & 7)
-                *reinterpret_cast<uint32_t*>(ds_row + rs * 1024 + (((piece0 + k) ^ tr) << 4)) =
+                // 8-row groups are 1024 bytes apart; 16-byte piece k of a row sits at position k ^ (row & 7)
+                *reinterpret_cast<uint32_t*>(ds_row + rs * 1024 + ((k ^ tr) << 4)) =
                     (MODE == 1 && c_hi[hl * 2 + rs] <= 0) ? 0u : ds_pack[2 * k + rs];
             }
         }
-        const uint32_t t = hl == 0 ? ta : tb;
-        tmem_st_16x128b_x4(t + COL_ST + c0, p_pack);
-        tmem_st_16x128b_x4(t + COL_DPT + c0, ds_pack);
+        tmem_st_16x128b_x8(taddr + COL_ST + cbase, p_pack);
+        tmem_st_16x128b_x8(taddr + COL_DPT + cbase, ds_pack);
     }
 }
 
@@ -240,7 +235,7 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
         for (int h = 0; h < 2; ++h) {
             mbar_init(&sm.s_full[h], 1);
-            mbar_init(&sm.p_full[h], NUM_COMPUTE_THREADS);
+            mbar_init(&sm.p_full[h], NUM_COMPUTE_THREADS / 2);
         }
         mbar_init(&sm.dq_full, 1);
         mbar_init(&sm.dq_empty, 128);
@@ -412,11 +407,11 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
                     if (ks < nk)
-                        mma_ts(tmem + COL_DV, tmem + COL_ST + h * HQ + ks * 8 + (ks >> 1) * 16, dod + ks * 128, idesc_acc, !first || (ks > 0));
+                        mma_ts(tmem + COL_DV, tmem + COL_ST + h * HQ + ks * 8, dod + ks * 128, idesc_acc, !first || (ks > 0));
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks)
                     if (ks < nk)
-                        mma_ts(tmem + COL_DK, tmem + COL_DPT + h * HQ + ks * 8 + (ks >> 1) * 16, qd + ks * 128, idesc_acc, !first || (ks > 0));
+                        mma_ts(tmem + COL_DK, tmem + COL_DPT + h * HQ + ks * 8, qd + ks * 128, idesc_acc, !first || (ks > 0));
             };
 
             auto wait1 = [&](uint64_t* a, uint32_t pa, int code) -> bool {
@@ -649,12 +644,12 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         // ================================================================== compute warpgroups
         reg_inc<REGS_COMPUTE>();
         const int quarter = warp & 3;
-        const int wg = warp >> 2;                           // this warpgroup's 32 columns of every 64-query buffer
+        const int h = warp >> 2;                            // the half of every step this warpgroup owns
         const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
         const float sl2 = args.scale_log2;
         bool ok = true;
         int gs = 0;                                         // steps seen so far (aux ring, dS buffer parity)
-        int nsh[2] = {0, 0};                                // non-empty buffers seen so far, per buffer of the step
+        int nsh = 0;                                        // non-empty halves of this warpgroup seen so far
 
         for (int g = item_begin; g < item_end && ok; ++g) {
             const BwdWork w = get_work(g);
@@ -680,48 +675,42 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             for (int i = 0; i < n_steps && ok; ++i, ++gs) {
                 const int q0 = w.q_begin + i * BQ;
                 const int n_valid = min(BQ, w.q_end - q0);
+                const int n_cols = half_cols(w, i, h);
+                const int cbase = h * HQ;                   // first query column of this half inside the step
 
                 const int aslot = gs % AUX_STAGES;
                 ok = __all_sync(0xffffffffu, mbar_wait(&sm.aux_full[aslot], (gs / AUX_STAGES) & 1, abort_flag));
                 if (!ok) { if (lane == 0) report_timeout(args.status, 0x1500 + i); break; }
 
-                int c_lo[4] = {0, 0, 0, 0}, c_hi[4] = {0, 0, 0, 0};     // visible query columns of the four rows in this step
-                if (tile_masked) {
-#pragma unroll
-                    for (int r4 = 0; r4 < 4; ++r4) {
-                        c_lo[r4] = max(qlo[r4] - q0, 0);
-                        c_hi[r4] = min(qhi[r4] - q0, n_valid);
-                    }
-                }
-                // The step's two 64-query buffers in turn; in each, this warpgroup owns 32 columns.  While both
-                // warpgroups work on one buffer the tensor core consumes the other and refills it for the next step.
-#pragma unroll 1
-                for (int u = 0; u < 2 && ok; ++u) {
-                    const int n_cols = half_cols(w, i, u);
-                    if (n_cols == 0) continue;
-                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[u], nsh[u] & 1, abort_flag));
+                if (n_cols > 0) {
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[h], nsh & 1, abort_flag));
                     if (!ok) { if (lane == 0) report_timeout(args.status, 0x1580 + i); break; }
-                    ++nsh[u];
+                    ++nsh;
                     tc_fence_after();
-                    if (n_cols > wg * (HQ / 2)) {
-                        const int c0 = u * HQ + wg * (HQ / 2);
-                        // tiles whose rows all see every column skip the mask code
-                        if (!tile_masked)
-                            softmax_grad_cols<0>(lane_base, c0, wg * 4, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi,
-                                                 sm.ds[gs & 1][u], quarter, lane);
-                        else if (rows_only)
-                            softmax_grad_cols<1>(lane_base, c0, wg * 4, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi,
-                                                 sm.ds[gs & 1][u], quarter, lane);
+                    // tiles whose rows all see every column skip the mask code
+                    if (tile_masked) {
+                        int c_lo[4], c_hi[4];               // visible query columns of the four rows in this step
+#pragma unroll
+                        for (int r4 = 0; r4 < 4; ++r4) {
+                            c_lo[r4] = max(qlo[r4] - q0, 0);
+                            c_hi[r4] = min(qhi[r4] - q0, n_valid);
+                        }
+                        if (rows_only)
+                            softmax_grad_half<1>(lane_base, cbase, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi,
+                                                 sm.ds[gs & 1][h], quarter, lane);
                         else
-                            softmax_grad_cols<2>(lane_base, c0, wg * 4, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi,
-                                                 sm.ds[gs & 1][u], quarter, lane);
-                        tmem_st_wait();
-                        tc_fence_before();
-                        fence_proxy_async_smem();
+                            softmax_grad_half<2>(lane_base, cbase, sm.lse2[aslot], sm.delta[aslot], sl2, c_lo, c_hi,
+                                                 sm.ds[gs & 1][h], quarter, lane);
+                    } else {
+                        const int none[4] = {0, 0, 0, 0};
+                        softmax_grad_half<0>(lane_base, cbase, sm.lse2[aslot], sm.delta[aslot], sl2, none, none,
+                                                 sm.ds[gs & 1][h], quarter, lane);
                     }
-                    mbar_arrive(&sm.p_full[u]);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    fence_proxy_async_smem();
+                    mbar_arrive(&sm.p_full[h]);
                 }
-                if (!ok) break;
                 mbar_arrive(&sm.aux_empty[aslot]);      // this thread is done with the step's lse / delta
             }
         }
