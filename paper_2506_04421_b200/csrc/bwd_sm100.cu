@@ -725,14 +725,18 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------------
-// delta_i = sum_d dO_id * O_id  (one warp per 4 rows: 8 lanes x 16 bytes cover a row)
+// delta_i = sum_d dO_id * O_id  (one warp per 4 rows: 8 lanes x 16 bytes cover a row).  The same pass
+// clears the fp32 dQ accumulator (32 bytes per lane), which saves a separate pass over it.
 __global__ void __launch_bounds__(256)
 hmar_bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
-                      float* __restrict__ delta, size_t n_rows) {
+                      float* __restrict__ delta, float* __restrict__ dq_acc, size_t n_rows) {
     const size_t row = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
     const int part = threadIdx.x & 7;
     float acc = 0.f;
     if (row < n_rows) {
+        float4* z = reinterpret_cast<float4*>(dq_acc + row * D + part * 8);
+        z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+        z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
         const uint4 a = *reinterpret_cast<const uint4*>(out + row * D + part * 8);
         const uint4 b = *reinterpret_cast<const uint4*>(dout + row * D + part * 8);
         const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
@@ -788,13 +792,8 @@ cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUte
     if (e != cudaSuccess) return e;
     const size_t n_rows = (size_t)BH * args.L;
     {
-        KernelTimer timer("memset_dq_acc", stream);
-        e = cudaMemsetAsync(args.dq_acc, 0, n_rows * D * sizeof(float), stream);
-        if (e != cudaSuccess) return e;
-    }
-    {
         KernelTimer timer("hmar_bwd_delta_kernel", stream);
-        hmar_bwd_delta_kernel<<<(unsigned)((n_rows * 8 + 255) / 256), 256, 0, stream>>>(out, dout, args.delta_w, n_rows);
+        hmar_bwd_delta_kernel<<<(unsigned)((n_rows * 8 + 255) / 256), 256, 0, stream>>>(out, dout, args.delta_w, args.dq_acc, n_rows);
     }
     {
         KernelTimer timer("hmar_bwd_tc_kernel", stream);
