@@ -389,7 +389,9 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 const bool ra = mbar_try_wait(a, pa);
                 const bool rb = !have_b || mbar_try_wait(b, pb);
                 if (__all_sync(0xffffffffu, ra && rb)) return true;
-                const bool done = mbar_wait(a, pa, abort_flag) && (!have_b || mbar_wait(b, pb, abort_flag));
+                // a barrier seen complete is not looked at again: a look is a shared-memory round trip behind the
+                // compute warps' stores, on the critical path of the step
+                const bool done = (ra || mbar_wait(a, pa, abort_flag)) && (rb || mbar_wait(b, pb, abort_flag));
                 if (__all_sync(0xffffffffu, done)) return true;
                 if (lane == 0) report_timeout(args.status, code);
                 return false;
