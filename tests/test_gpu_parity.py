@@ -106,6 +106,37 @@ def test_large_logits_exercise_running_max():
     _run_training(_Wl((1, 2, 3, 4, 6, 9, 13, 18)), torch.float32, gain=8.0)
 
 
+def test_rows_past_a_partial_key_tile_cannot_reach_dq():
+    # Scale 2 has 81 keys: its key tile is loaded 128 rows high, so rows 81..127 hold the first keys of
+    # scale 3, which the tile's queries of scale 2 must not see.  Those keys are made 16 times larger
+    # (a power of two: still exact in bf16), so that a logit against them is worth e^40 and more: if such
+    # a row leaked into dQ = dS K the result would be off by many orders of magnitude.
+    wl = _Wl((1, 9, 13, 5))
+    q, k, v, do = training_inputs(wl, bf16=True)
+    n = [s * s for s in wl.side_lens]
+    k = k.copy()
+    k[:, n[0] + n[1]:n[0] + n[1] + n[2], :] *= 16.0
+    tq, tk, tv, tdo = (to_device(x, wl.B, wl.H, torch.bfloat16) for x in (q, k, v, do))
+    out, lse = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale)
+    ref_out, ref_lse = orc.attn_fwd(q, k, v, wl.side_lens, wl.softmax_scale)
+    _assert_close("out", out, ref_out, False)
+    _assert_lse(lse, ref_lse, False)
+    dq, dk, dv = hmar.hmar_attn_bwd(tq, tk, tv, out, lse, tdo, wl.side_lens, wl.softmax_scale)
+    rq, rk, rv = orc.attn_bwd(q, k, v, do, wl.side_lens, wl.softmax_scale)
+    assert torch.isfinite(dq).all() and torch.isfinite(dk).all() and torch.isfinite(dv).all()
+    # the queries that do see the large keys have logits of N(0, 16^2): tolerances as in the gain test
+    _assert_close("dq", dq, rq, False, 16.0)
+    _assert_close("dk", dk, rk, False, 16.0)
+    # dV_j = sum_i P_ij dO_i: with logits this large several queries put P close to 1 on the same key, and the
+    # bf16 roundings of those P (2^-9 relative, times |dO| up to 4) add up, so twice the usual bound here
+    _assert_close("dv", dv, rv, False, 2.0)
+    # the rows the test is about: queries of scale 2 see keys of scales 1 and 2 only, all of them O(1)
+    lo, hi = n[0], n[0] + n[1]
+    d = np.abs(dq.detach().double().cpu().numpy().reshape(rq.shape)[:, lo:hi] - rq[:, lo:hi])
+    assert d.max() <= BF16_MAX, f"dq of the tile's own queries: max abs err {d.max():.3e}"
+    _no_device_error()
+
+
 def test_fp32_debug_build_512_shape_one_head():
     _run_training(_Wl(CONFIGS["512_d24_train"].side_lens, B=1, H=1), torch.float32)
 
