@@ -255,14 +255,17 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     const int n = half_cols(nv, h), n_next = half_cols(nv_next, h);
-                    // one burst: O_h += P_h V_h of tile j, then S_h of tile j + 1 over the columns P_h leaves
-                    if (n > 0) {
-                        ok = wait(&sm.p_full[h], par_p[h], 0x600 + j);
-                        par_p[h] ^= 1;
-                    }
-                    if (ok && h == 0) {
+                    // one burst: O_h += P_h V_h of tile j, then S_h of tile j + 1 over the columns P_h leaves.
+                    // The copies are looked at first (normally long complete): a look at a barrier is a
+                    // shared-memory round trip behind the softmax warps' traffic, and after the softmax
+                    // warpgroup's arrival every such trip delays the products it is waiting for.
+                    if (h == 0) {
                         ok = wait(&sm.v_full[slot], (j / NSTAGE) & 1, 0x500 + j);
                         if (ok && more) ok = wait(&sm.k_full[slot_next], ((j + 1) / NSTAGE) & 1, 0x400 + j);
+                    }
+                    if (ok && n > 0) {
+                        ok = wait(&sm.p_full[h], par_p[h], 0x600 + j);
+                        par_p[h] ^= 1;
                     }
                     if (!ok) break;
                     tc_fence_after();
