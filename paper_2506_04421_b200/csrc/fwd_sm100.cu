@@ -148,6 +148,15 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         mbar_init(&sm.o_done, 1);
         mbar_init(&sm.stats_ready, NUM_SOFTMAX_THREADS);
         fence_mbar_init();
+        // The block's first copies (Q, first K and V tiles) start here, before the TMEM allocation and the
+        // block-wide barrier, so that their latency overlaps the rest of the set-up.
+        const KvTile t0 = kv_tile(w, tiles0, 0);
+        mbar_arrive_expect_tx(&sm.q_full, TILE_BYTES);
+        tma_load_3d(sm.q, &map_q, &sm.q_full, 0, w.row_begin, bh);
+        mbar_arrive_expect_tx(&sm.k_full[0], TILE_BYTES);
+        tma_load_3d(sm.k[0], t0.seg ? &map_k1 : &map_k0, &sm.k_full[0], 0, t0.coord, bh);
+        mbar_arrive_expect_tx(&sm.v_full[0], TILE_BYTES);
+        tma_load_3d(sm.v[0], t0.seg ? &map_v1 : &map_v0, &sm.v_full[0], 0, t0.coord, bh);
     }
     if (warp == MMA_WARP) {
         tmem_alloc(&sm.tmem_base, TMEM_COLS);
@@ -170,12 +179,10 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 prefetch_tensormap(&map_q);
                 prefetch_tensormap(&map_k0);
                 prefetch_tensormap(&map_v0);
-                mbar_arrive_expect_tx(&sm.q_full, TILE_BYTES);
-                tma_load_3d(sm.q, &map_q, &sm.q_full, 0, w.row_begin, bh);
             }
             __syncwarp();
             bool ok = true;
-            for (int j = 0; j < n_tiles && ok; ++j) {
+            for (int j = 1; j < n_tiles && ok; ++j) {           // tile 0 was requested during the set-up
                 const int slot = j % NSTAGE;
                 const uint32_t par = ((j / NSTAGE) & 1) ^ 1;     // parity of the previous use of the slot
                 const KvTile t = kv_tile(w, tiles0, j);
