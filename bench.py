@@ -32,7 +32,7 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
 # The captures are of the batch-4 case (traffic grows in proportion to the heads), scaled by 4 to the full batch.
-NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (234_195_968 + 117_513_728), "hmar_fwd": 4 * (82_638_336 + 10_579_200)}
+NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (236_007_680 + 119_998_976), "hmar_fwd": 4 * (82_653_440 + 12_209_152)}
 
 
 def pairs_per_head(side_lens):
