@@ -32,7 +32,7 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
 # The captures are of the batch-4 case (traffic grows in proportion to the heads), scaled by 4 to the full batch.
-NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (236_007_680 + 119_998_976), "hmar_fwd": 4 * (82_653_440 + 12_209_152)}
+NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (234_428_160 + 117_550_336), "hmar_fwd": 4 * (82_650_624 + 11_561_472)}
 
 
 def pairs_per_head(side_lens):
@@ -202,6 +202,32 @@ def time_training_shape(hmar, wl_x, dev, window, reps=3):
     return f_ms, b_ms
 
 
+def time_packed_forward(hmar, wl_x, dev, reps=5):
+    """ms of the forward on the packed projection output [B,L,3,H,D] -> [B,L,H,D], and of the copies that the
+    contiguous entry point would need around it for the same data (context leg)."""
+    import torch
+    from workloads.device import bulk_normal
+    B, H, L, D = wl_x.B, wl_x.H, wl_x.L, wl_x.D
+    qkv = bulk_normal(wl_x.seed, 9, B, L, 3 * H, D, torch.bfloat16, dev).view(B, L, 3, H, D)
+    out = torch.empty((B, L, H, D), dtype=torch.bfloat16, device=dev)
+    lse = torch.empty((B, H, L), dtype=torch.float32, device=dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    p_ms = c_ms = 0.0
+    for it in range(reps + 1):
+        ev[0].record()
+        hmar.hmar_attn_fwd_packed(qkv, wl_x.side_lens, wl_x.softmax_scale, out=out, lse=lse)
+        ev[1].record()
+        q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3).contiguous() for i in range(3))
+        o = torch.empty_like(q)
+        o.permute(0, 2, 1, 3).contiguous()
+        ev[2].record()
+        torch.cuda.synchronize()
+        if it:
+            p_ms += ev[0].elapsed_time(ev[1]) / reps
+            c_ms += ev[1].elapsed_time(ev[2]) / reps
+    return p_ms, c_ms
+
+
 def run_reference(args, wl):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -311,6 +337,11 @@ def run_ours(args, wl):
             extras["block_causal_same_kernels"] = {"fwd_ms": round(cf, 4), "bwd_ms": round(cb, 4),
                                                    "markov_speedup_fwd": round(cf / fwd_ms, 3),
                                                    "markov_speedup_bwd": round(cb / bwd_ms, 3)}
+            torch.cuda.empty_cache()
+            # forward on the packed QKV projection output, and the transposing copies it makes unnecessary
+            pk, cp = time_packed_forward(hmar, wl, dev)
+            extras["packed_qkv_forward"] = {"fwd_ms": round(pk, 4), "transposes_avoided_ms": round(cp, 4),
+                                            "layout": "qkv [B,L,3,H,D] -> out [B,L,H,D]"}
             torch.cuda.empty_cache()
             # 1024 x 1024 (synthetic 14-scale schedule ending at 64 x 64, L = 9451), Markov mask
             wl_big = CONFIGS["1024_d24_train"]

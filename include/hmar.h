@@ -69,6 +69,16 @@ int hmar_attn_fwd_f32(const float* q, const float* k, const float* v, float* out
                       int B, int H, int D, int n_scales, const int* side_lens,
                       float softmax_scale, void* stream);
 
+/* Training forward on the packed output of the QKV projection (Sec. 4.1: the kernel sits between the
+ * transformer block's QKV projection and its output projection; reading the projection's layout saves the
+ * transposing copies around the kernel).  bf16 only, Markovian mask.
+ *   qkv : [B,L,3,H,D] in (q, k, v of a token side by side);  out : [B,L,H,D] out (the layout the output
+ *   projection reads);  lse : [B,H,L] fp32 out, as for hmar_attn_fwd (the backward takes contiguous
+ *   [B,H,L,D] tensors only).  All pointers device, 16-byte aligned.  HMAR_ERR_UNSUPPORTED while the
+ *   fall-back kernels are forced (they read contiguous tensors only); other errors as for hmar_attn_fwd. */
+int hmar_attn_fwd_packed(const void* qkv, void* out, float* lse, int B, int H, int D, int n_scales,
+                         const int* side_lens, float softmax_scale, void* stream);
+
 /* The same forward under another block mask of the same family (see hmar_window).  Everything else -
  * layouts, lse convention, precision, errors - is as for hmar_attn_fwd; an unknown `window` is
  * HMAR_ERR_BAD_ARG. */

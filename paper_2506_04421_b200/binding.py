@@ -26,7 +26,7 @@ HMAR_WINDOW_CAUSAL = 1      # scales 1..k (VAR's block-causal mask)
 HMAR_WINDOW_SELF = 2        # scale k only (block-diagonal)
 
 EXPORTED_SYMBOLS = (
-    "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_fwd_window", "hmar_attn_fwd_window_f32",
+    "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_fwd_window", "hmar_attn_fwd_window_f32", "hmar_attn_fwd_packed",
     "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd", "hmar_attn_bwd_f32", "hmar_attn_bwd_window",
     "hmar_attn_bwd_window_f32", "hmar_schedule_tiles_window", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_schedule_tiles",
     "hmar_device_status", "hmar_profile_begin", "hmar_profile_end", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
@@ -55,6 +55,7 @@ def lib():
     L.hmar_attn_fwd_f32.argtypes = L.hmar_attn_fwd.argtypes
     L.hmar_attn_fwd_window.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, ip, i, fp, vp]
     L.hmar_attn_fwd_window_f32.argtypes = L.hmar_attn_fwd_window.argtypes
+    L.hmar_attn_fwd_packed.argtypes = [vp, vp, vp, i, i, i, i, ip, fp, vp]
     L.hmar_attn_bwd_workspace_bytes.argtypes = [i, i, i, i, ip]
     L.hmar_attn_bwd_workspace_bytes.restype = ctypes.c_size_t
     L.hmar_attn_bwd.argtypes = [vp] * 9 + [vp, ctypes.c_size_t, i, i, i, i, ip, fp, vp]
@@ -137,6 +138,23 @@ def hmar_attn_fwd(q, k, v, side_lens, softmax_scale, out=None, lse=None, stream=
     fn = lib().hmar_attn_fwd_f32 if _is_f32(q) else lib().hmar_attn_fwd
     _check(fn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), B, H, D, n, sides,
               float(softmax_scale), _stream(stream)), "hmar_attn_fwd")
+    return out, lse
+
+
+def hmar_attn_fwd_packed(qkv, side_lens, softmax_scale, out=None, lse=None, stream=None):
+    """Training forward on the packed projection output. qkv: [B,L,3,H,D] bf16.
+    Returns (out [B,L,H,D], lse [B,H,L] fp32)."""
+    _need(qkv, out, lse)
+    B, L, three, H, D = qkv.shape
+    if three != 3:
+        raise ValueError("qkv must be [B, L, 3, H, D]")
+    if out is None:
+        out = torch.empty((B, L, H, D), dtype=qkv.dtype, device=qkv.device)
+    if lse is None:
+        lse = torch.empty((B, H, L), dtype=torch.float32, device=qkv.device)
+    sides, n = _sides(side_lens)
+    _check(lib().hmar_attn_fwd_packed(_ptr(qkv), _ptr(out), _ptr(lse), B, H, D, n, sides, float(softmax_scale),
+                                      _stream(stream)), "hmar_attn_fwd_packed")
     return out, lse
 
 

@@ -207,6 +207,23 @@ int hmar_attn_fwd_window_f32(const float* q, const float* k, const float* v, flo
     return fwd_impl<float>(q, k, v, out, lse, B, H, D, n_scales, side_lens, window, softmax_scale, stream, false);
 }
 
+int hmar_attn_fwd_packed(const void* qkv, void* out, float* lse, int B, int H, int D, int n_scales,
+                         const int* side_lens, float softmax_scale, void* stream) {
+    int rc = check_shape(B, H, D);
+    if (rc != HMAR_OK) return rc;
+    ScaleTable st;
+    rc = check_sides(n_scales, side_lens, HMAR_WINDOW_MARKOV, &st);
+    if (rc != HMAR_OK) return rc;
+    if (check_scale(softmax_scale) != HMAR_OK) return HMAR_ERR_BAD_ARG;
+    if (!qkv || !out || !lse) return HMAR_ERR_BAD_ARG;
+    if (!aligned16(qkv) || !aligned16(out) || !aligned16(lse)) return HMAR_ERR_BAD_ARG;
+    rc = check_device();
+    if (rc != HMAR_OK) return rc;
+    if (g_force_simt.load()) return HMAR_ERR_UNSUPPORTED;      // the fall-back kernels read contiguous tensors only
+    return tc_fwd_packed((const bf16*)qkv, (bf16*)out, lse, B, H, st, softmax_scale, device_status_ptr(),
+                         static_cast<cudaStream_t>(stream));
+}
+
 int hmar_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse, int B, int H, int D,
                   int n_scales, const int* side_lens, float softmax_scale, void* stream) {
     return hmar_attn_fwd_window(q, k, v, out, lse, B, H, D, n_scales, side_lens, HMAR_WINDOW_MARKOV, softmax_scale, stream);

@@ -117,6 +117,7 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     // ---- which tile of which head
     const int bh = blockIdx.x / args.n_work;
     const int wi = blockIdx.x % args.n_work;
+    const int batch = bh / args.heads_per_batch, head = bh - batch * args.heads_per_batch;
     FwdWork w;
     if (args.work != nullptr) {
         w = args.work[wi];
@@ -152,11 +153,11 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         // block-wide barrier, so that their latency overlaps the rest of the set-up.
         const KvTile t0 = kv_tile(w, tiles0, 0);
         mbar_arrive_expect_tx(&sm.q_full, TILE_BYTES);
-        tma_load_3d(sm.q, &map_q, &sm.q_full, 0, w.row_begin, bh);
+        tma_load_4d(sm.q, &map_q, &sm.q_full, 0, w.row_begin, head, batch);
         mbar_arrive_expect_tx(&sm.k_full[0], TILE_BYTES);
-        tma_load_3d(sm.k[0], t0.seg ? &map_k1 : &map_k0, &sm.k_full[0], 0, t0.coord, bh);
+        tma_load_4d(sm.k[0], t0.seg ? &map_k1 : &map_k0, &sm.k_full[0], 0, t0.coord, head, batch);
         mbar_arrive_expect_tx(&sm.v_full[0], TILE_BYTES);
-        tma_load_3d(sm.v[0], t0.seg ? &map_v1 : &map_v0, &sm.v_full[0], 0, t0.coord, bh);
+        tma_load_4d(sm.v[0], t0.seg ? &map_v1 : &map_v0, &sm.v_full[0], 0, t0.coord, head, batch);
     }
     if (warp == MMA_WARP) {
         tmem_alloc(&sm.tmem_base, TMEM_COLS);
@@ -190,14 +191,14 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 if (!ok) { if (lane == 0) report_timeout(args.status, 0x100 + j); break; }
                 if (leader) {
                     mbar_arrive_expect_tx(&sm.k_full[slot], TILE_BYTES);
-                    tma_load_3d(sm.k[slot], t.seg ? &map_k1 : &map_k0, &sm.k_full[slot], 0, t.coord, bh);
+                    tma_load_4d(sm.k[slot], t.seg ? &map_k1 : &map_k0, &sm.k_full[slot], 0, t.coord, head, batch);
                 }
                 __syncwarp();
                 if (j >= NSTAGE) ok = __all_sync(0xffffffffu, mbar_wait(&sm.v_empty[slot], par, abort_flag));
                 if (!ok) { if (lane == 0) report_timeout(args.status, 0x200 + j); break; }
                 if (leader) {
                     mbar_arrive_expect_tx(&sm.v_full[slot], TILE_BYTES);
-                    tma_load_3d(sm.v[slot], t.seg ? &map_v1 : &map_v0, &sm.v_full[slot], 0, t.coord, bh);
+                    tma_load_4d(sm.v[slot], t.seg ? &map_v1 : &map_v0, &sm.v_full[slot], 0, t.coord, head, batch);
                 }
                 __syncwarp();
             }
@@ -434,7 +435,8 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             tmem_ld32(lane_base + COL_O + HN + h * 32, b1);            // O_b
             tmem_ld_wait();
             if (row_ok) {
-                __nv_bfloat16* orow = args.out + ((size_t)bh * args.n_q_rows + row) * D + h * 32;
+                __nv_bfloat16* orow = args.out + batch * args.out_batch_stride + head * args.out_head_stride +
+                                      row * args.out_row_stride + h * 32;
                 uint4* dst = reinterpret_cast<uint4*>(orow);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {

@@ -21,6 +21,8 @@ struct FwdArgs {
     const FwdWork* work;     // n_work tiles per head; nullptr = inference step (tiles derived in-kernel)
     int n_work;
     int n_q_rows;            // rows per head of q / out / lse
+    int heads_per_batch;     // H: head bh is head bh % H of batch bh / H (the tensor maps are 4-D: D, rows, H, B)
+    long long out_row_stride, out_head_stride, out_batch_stride;   // of `out`, in elements (lse is always [B*H, rows])
     int n0, n1;              // inference step: rows of the previous / current scale's keys
     float scale_log2;        // softmax_scale * log2(e)
     __nv_bfloat16* out;

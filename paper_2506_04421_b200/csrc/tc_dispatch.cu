@@ -51,6 +51,21 @@ static bool make_rows_map(CUtensorMap* map, const void* base, int heads, int row
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 4-D map (64 elements, rows, heads, batches) with the strides of the tensor in elements; boxes of 128 rows
+// of one head.  Serves the contiguous [B, H, rows, 64] layout and a packed [B, rows, 3, H, 64] one alike.
+static bool make_rows_map4(CUtensorMap* map, const void* base, int batches, int heads, int rows, long long row_stride,
+                           long long head_stride, long long batch_stride) {
+    EncodeTiledFn fn = encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows, (cuuint64_t)heads, (cuuint64_t)batches};
+    const cuuint64_t strides[3] = {(cuuint64_t)row_stride * 2, (cuuint64_t)head_stride * 2, (cuuint64_t)batch_stride * 2};
+    const cuuint32_t box[4] = {(cuuint32_t)kHeadDim, (cuuint32_t)kTileRows, 1, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Tensor map of the fp32 dQ accumulator seen as [rows, 64]: boxes of 32 rows x 32 columns (128 bytes,
 // 128-byte swizzle), the unit in which a warp of the backward kernel adds dQ pieces to it.
 static bool make_acc_map(CUtensorMap* map, const float* base, size_t rows) {
@@ -153,18 +168,25 @@ void tc_release_plans() {
 }
 
 // ------------------------------------------------------------------------------------------------
-int tc_fwd(const bf16* q, const bf16* k, const bf16* v, bf16* out, float* lse, int BH, const ScaleTable& st,
-           float scale, int* status, cudaStream_t stream) {
+// Forward on tensors whose layout is given by strides (elements): q, k, v share one layout, out has its own.
+static int tc_fwd_strided(const bf16* q, const bf16* k, const bf16* v, bf16* out, float* lse, int B, int H,
+                          const ScaleTable& st, float scale, long long in_row, long long in_head, long long in_batch,
+                          long long out_row, long long out_head, long long out_batch, int* status, cudaStream_t stream) {
     const Plan* plan = get_plan(st);
     if (plan == nullptr) return HMAR_ERR_CUDA;
     const int L = st.start[st.n_scales];
     CUtensorMap mq, mk, mv;
-    if (!make_rows_map(&mq, q, BH, L) || !make_rows_map(&mk, k, BH, L) || !make_rows_map(&mv, v, BH, L))
+    if (!make_rows_map4(&mq, q, B, H, L, in_row, in_head, in_batch) || !make_rows_map4(&mk, k, B, H, L, in_row, in_head, in_batch) ||
+        !make_rows_map4(&mv, v, B, H, L, in_row, in_head, in_batch))
         return HMAR_ERR_CUDA;
     FwdArgs a{};
     a.work = plan->fwd_work;
     a.n_work = plan->n_fwd;
     a.n_q_rows = L;
+    a.heads_per_batch = H;
+    a.out_row_stride = out_row;
+    a.out_head_stride = out_head;
+    a.out_batch_stride = out_batch;
     a.n0 = L;
     a.n1 = 0;
     a.scale_log2 = scale * 1.4426950408889634f;
@@ -172,19 +194,35 @@ int tc_fwd(const bf16* q, const bf16* k, const bf16* v, bf16* out, float* lse, i
     a.lse = lse;
     a.status = status;
     a.st = st;
-    return launch_fwd_tc(mq, mk, mv, mk, mv, a, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
+    return launch_fwd_tc(mq, mk, mv, mk, mv, a, B * H, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
+}
+
+// Contiguous [B*H, L, 64] tensors: one "batch" of BH heads.
+int tc_fwd(const bf16* q, const bf16* k, const bf16* v, bf16* out, float* lse, int BH, const ScaleTable& st,
+           float scale, int* status, cudaStream_t stream) {
+    const long long L = st.start[st.n_scales];
+    return tc_fwd_strided(q, k, v, out, lse, 1, BH, st, scale, kHeadDim, L * kHeadDim, (long long)BH * L * kHeadDim,
+                          kHeadDim, L * kHeadDim, (long long)BH * L * kHeadDim, status, stream);
+}
+
+// Packed projection output qkv [B, L, 3, H, 64] (q, k, v of a token side by side), out [B, L, H, 64].
+int tc_fwd_packed(const bf16* qkv, bf16* out, float* lse, int B, int H, const ScaleTable& st, float scale, int* status,
+                  cudaStream_t stream) {
+    const long long L = st.start[st.n_scales], HD = (long long)H * kHeadDim;
+    return tc_fwd_strided(qkv, qkv + HD, qkv + 2 * HD, out, lse, B, H, st, scale, 3 * HD, kHeadDim, L * 3 * HD,
+                          HD, kHeadDim, L * HD, status, stream);
 }
 
 int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const bf16* k_cur, const bf16* v_cur,
                   bf16* out, float* lse, int BH, int n_prev, int n_cur, float scale, int* status,
                   cudaStream_t stream) {
     CUtensorMap mq, mk0, mv0, mk1, mv1;
-    if (!make_rows_map(&mq, q, BH, n_cur) || !make_rows_map(&mk1, k_cur, BH, n_cur) ||
-        !make_rows_map(&mv1, v_cur, BH, n_cur))
-        return HMAR_ERR_CUDA;
+    auto rows_map = [&](CUtensorMap* m, const bf16* base, int rows) {
+        return make_rows_map4(m, base, 1, BH, rows, kHeadDim, (long long)rows * kHeadDim, (long long)BH * rows * kHeadDim);
+    };
+    if (!rows_map(&mq, q, n_cur) || !rows_map(&mk1, k_cur, n_cur) || !rows_map(&mv1, v_cur, n_cur)) return HMAR_ERR_CUDA;
     if (n_prev > 0) {
-        if (!make_rows_map(&mk0, k_prev, BH, n_prev) || !make_rows_map(&mv0, v_prev, BH, n_prev))
-            return HMAR_ERR_CUDA;
+        if (!rows_map(&mk0, k_prev, n_prev) || !rows_map(&mv0, v_prev, n_prev)) return HMAR_ERR_CUDA;
     } else {
         mk0 = mk1;
         mv0 = mv1;
@@ -193,6 +231,10 @@ int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const b
     a.work = nullptr;
     a.n_work = (n_cur + kTileRows - 1) / kTileRows;
     a.n_q_rows = n_cur;
+    a.heads_per_batch = BH;
+    a.out_row_stride = kHeadDim;
+    a.out_head_stride = (long long)n_cur * kHeadDim;
+    a.out_batch_stride = (long long)BH * n_cur * kHeadDim;
     a.n0 = n_prev;
     a.n1 = n_cur;
     a.scale_log2 = scale * 1.4426950408889634f;

@@ -137,6 +137,28 @@ def test_rows_past_a_partial_key_tile_cannot_reach_dq():
     _no_device_error()
 
 
+@pytest.mark.parametrize("sides,B,H", [((1, 2, 3, 4, 6, 9, 13), 2, 3), ((3, 11), 1, 2), ((16, 3, 17), 3, 1)])
+def test_packed_qkv_forward(sides, B, H):
+    # qkv [B, L, 3, H, D] (the projection's layout), out [B, L, H, D]; the oracle sees the same values as
+    # [B*H, L, D] tensors
+    wl = _Wl(sides, B=B, H=H)
+    q, k, v = training_inputs(wl, bf16=True, with_dout=False)
+    L, D = wl.L, wl.D
+    packed = np.stack([x.reshape(B, H, L, D) for x in (q, k, v)], axis=0)          # [3, B, H, L, D]
+    packed = np.ascontiguousarray(packed.transpose(1, 3, 0, 2, 4))                 # [B, L, 3, H, D]
+    t = torch.from_numpy(packed).to(device="cuda", dtype=torch.bfloat16)
+    out, lse = hmar.hmar_attn_fwd_packed(t, wl.side_lens, wl.softmax_scale)
+    assert out.shape == (B, L, H, D) and lse.shape == (B, H, L)
+    ref_out, ref_lse = orc.attn_fwd(q, k, v, wl.side_lens, wl.softmax_scale)
+    _assert_close("out", out.permute(0, 2, 1, 3).contiguous(), ref_out, False)
+    _assert_lse(lse, ref_lse, False)
+    # the same values through the contiguous entry point give the same bits
+    tq, tk, tv = (to_device(x, B, H, torch.bfloat16) for x in (q, k, v))
+    out_c, lse_c = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale)
+    assert torch.equal(out_c, out.permute(0, 2, 1, 3)) and torch.equal(lse_c, lse)
+    _no_device_error()
+
+
 def test_fp32_debug_build_512_shape_one_head():
     _run_training(_Wl(CONFIGS["512_d24_train"].side_lens, B=1, H=1), torch.float32)
 

@@ -107,6 +107,18 @@ def test_argument_errors_are_reported_before_any_launch():
     assert f(p, p, p, p, p, p, None, 1, 1, 64, 2, 0, 0.125, None) == hmar.HMAR_ERR_BAD_ARG
 
 
+def test_packed_forward_argument_errors():
+    vp = ctypes.c_void_p
+    f = hmar.lib().hmar_attn_fwd_packed
+    p = vp(1 << 12)
+    sides = (ctypes.c_int * 2)(1, 2)
+    assert f(None, p, p, 1, 1, 64, 2, sides, 0.125, None) == hmar.HMAR_ERR_BAD_ARG
+    assert f(vp((1 << 12) + 2), p, p, 1, 1, 64, 2, sides, 0.125, None) == hmar.HMAR_ERR_BAD_ARG
+    assert f(p, p, p, 1, 1, 32, 2, sides, 0.125, None) == hmar.HMAR_ERR_UNSUPPORTED
+    assert f(p, p, p, 1, 1, 64, 0, sides, 0.125, None) == hmar.HMAR_ERR_BAD_ARG
+    assert f(p, p, p, 1, 1, 64, 2, sides, -1.0, None) == hmar.HMAR_ERR_BAD_ARG
+
+
 def test_valid_call_without_a_device_fails_loudly():
     import torch
     if torch.cuda.is_available():
