@@ -244,7 +244,12 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 o_started[h] = true;
             };
 
-            bool ok = wait(&sm.q_full, 0, 0x300) && wait(&sm.k_full[0], 0, 0x400);
+            bool ok = true;
+            {
+                const bool rq = mbar_try_wait(&sm.q_full, 0), rk = mbar_try_wait(&sm.k_full[0], 0);
+                if (!__all_sync(0xffffffffu, rq && rk))
+                    ok = (rq || wait(&sm.q_full, 0, 0x300)) && (rk || wait(&sm.k_full[0], 0, 0x400));
+            }
             if (ok) {
                 tc_fence_after();
                 const int nv = kv_tile(w, tiles0, 0).n_valid;
@@ -268,8 +273,12 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     // shared-memory round trip behind the softmax warps' traffic, and after the softmax
                     // warpgroup's arrival every such trip delays the products it is waiting for.
                     if (h == 0) {
-                        ok = wait(&sm.v_full[slot], (j / NSTAGE) & 1, 0x500 + j);
-                        if (ok && more) ok = wait(&sm.k_full[slot_next], ((j + 1) / NSTAGE) & 1, 0x400 + j);
+                        // both looks are sent before either answer is used
+                        const bool rv = mbar_try_wait(&sm.v_full[slot], (j / NSTAGE) & 1);
+                        const bool rk = !more || mbar_try_wait(&sm.k_full[slot_next], ((j + 1) / NSTAGE) & 1);
+                        if (!__all_sync(0xffffffffu, rv && rk))
+                            ok = (rv || wait(&sm.v_full[slot], (j / NSTAGE) & 1, 0x500 + j)) &&
+                                 (rk || wait(&sm.k_full[slot_next], ((j + 1) / NSTAGE) & 1, 0x400 + j));
                     }
                     if (ok && n > 0) {
                         ok = wait(&sm.p_full[h], par_p[h], 0x600 + j);
@@ -409,15 +418,16 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
 
         // ---- merge of the two halves and epilogue: this warpgroup writes output columns [32 h, 32 h + 32)
-        if (ok) {
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_done, 0, abort_flag));
-            if (!ok && lane == 0) report_timeout(args.status, 0xA00);
-        }
+        // (the row statistics are final once the last P is out: they are exchanged while the last products run)
         if (ok) {
             sm.stats[h][r] = make_float2(m_used, l);
             mbar_arrive(&sm.stats_ready);
             ok = __all_sync(0xffffffffu, mbar_wait(&sm.stats_ready, 0, abort_flag));
             if (!ok && lane == 0) report_timeout(args.status, 0xB00);
+        }
+        if (ok) {
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_done, 0, abort_flag));
+            if (!ok && lane == 0) report_timeout(args.status, 0xA00);
         }
         if (ok) {
             tc_fence_after();
