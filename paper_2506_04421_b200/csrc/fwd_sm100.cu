@@ -13,7 +13,11 @@
 //               running maximum is kept unless the tile exceeds it by more than 2^8 (then O_a and the
 //               row sum are rescaled first), P = 2^(s - m) goes back to TMEM as bf16 over S
 //   warps 4-7   the same for half b
-//   warp 8      TMA producer: Q once, then K and V tiles of 128 keys through a shared-memory ring
+//   warp 8      TMA producer: K and V tiles of 128 keys through a shared-memory ring (Q and the first K, V
+//               tiles are requested by thread 0 during the set-up).  The tensor maps are 4-D (64, rows,
+//               heads, batches) with the tensor's own strides, so contiguous [B,H,L,64] tensors and the
+//               packed [B,L,3,H,64] projection output go through the same code; the output address is
+//               formed from three strides
 //   warp 9      issues tcgen05.mma: S_x = Q K_x^T (both operands in shared memory), O_x += P_x V_x (P_x from
 //               TMEM, V_x an MN-major shared-memory operand), one burst per half and tile:
 //               O_x += P_x V_x of tile j, then S_x of tile j + 1 into the columns P_x has just left
