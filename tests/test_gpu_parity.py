@@ -159,6 +159,19 @@ def test_packed_qkv_forward(sides, B, H):
     _no_device_error()
 
 
+def test_packed_qkv_forward_full_size_matches_contiguous_bits():
+    # the headline shape as bench.py's packed leg runs it: the packed entry point must give the very bits
+    # of the contiguous one (which the sampled-head tests compare with the oracle at this size)
+    wl = CONFIGS["512_d24_train"]
+    B, H, L, D = wl.B, wl.H, wl.L, wl.D
+    qkv = bulk_normal(wl.seed, 9, B, L, 3 * H, D, torch.bfloat16, "cuda").view(B, L, 3, H, D)
+    out, lse = hmar.hmar_attn_fwd_packed(qkv, wl.side_lens, wl.softmax_scale)
+    q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3).contiguous() for i in range(3))
+    out_c, lse_c = hmar.hmar_attn_fwd(q, k, v, wl.side_lens, wl.softmax_scale)
+    assert torch.equal(out_c, out.permute(0, 2, 1, 3)) and torch.equal(lse_c, lse)
+    _no_device_error()
+
+
 def test_fp32_debug_build_512_shape_one_head():
     _run_training(_Wl(CONFIGS["512_d24_train"].side_lens, B=1, H=1), torch.float32)
 
