@@ -56,6 +56,7 @@ constexpr int NSTAGE = 3;
 constexpr int AUX_STAGES = 8;        // ring of lse / delta rows, loaded this many steps ahead
 constexpr int TILE_BYTES = 128 * D * 2;          // 16 KB
 constexpr int WORK_CACHE = 64;       // work tiles of a head kept in shared memory
+constexpr int MAX_CHUNKS = 64;       // runs of consecutive items a block can be given
 constexpr int NUM_COMPUTE_THREADS = 256;
 constexpr int DRAIN_WARP0 = 8, PRODUCER_WARP = 12, MMA_WARP = 13, AUX_WARP = 14;
 constexpr int NUM_THREADS = 512;
@@ -85,7 +86,10 @@ struct __align__(1024) SharedStorage {
     BwdWork work[WORK_CACHE];               // the head's work list (its first WORK_CACHE tiles)
     uint32_t tmem_base;
     int abort_flag;
-    int item_begin, item_end;
+    // The block's items: n_chunks runs of consecutive items; run c starts at item chunk_item[c] and holds the
+    // block's items number chunk_first[c] .. chunk_first[c + 1] - 1.
+    int chunk_item[MAX_CHUNKS], chunk_first[MAX_CHUNKS + 1];
+    int n_chunks;
 };
 
 __device__ __forceinline__ void report_timeout(int* status, int where) {
@@ -208,6 +212,9 @@ __device__ __forceinline__ int first_item_at_cost(const BwdArgs& args, long long
     return (int)head * args.n_work + lo;
 }
 
+// CHUNKED: the block's items are several runs (long sequences, see the launcher); otherwise one contiguous run,
+// and the item loops compile to plain counting.
+template <bool CHUNKED>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
@@ -248,10 +255,30 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         mbar_init(&sm.acc_full, 1);
         mbar_init(&sm.acc_empty, 128);
         fence_mbar_init();
-        const long long total = (long long)args.n_heads * args.head_cost;
-        sm.item_begin = first_item_at_cost(args, total * blockIdx.x / gridDim.x);
-        sm.item_end = blockIdx.x + 1 == gridDim.x ? args.n_heads * n_work
-                                                  : first_item_at_cost(args, total * (blockIdx.x + 1) / gridDim.x);
+        int nch = 0, cnt = 0;
+        if (!CHUNKED) {
+            // one run: a contiguous stretch of the item list of about 1 / gridDim.x of the total cost
+            const long long total = (long long)args.n_heads * args.head_cost;
+            const int ib = first_item_at_cost(args, total * blockIdx.x / gridDim.x);
+            const int ie = blockIdx.x + 1 == gridDim.x ? args.n_heads * n_work
+                                                       : first_item_at_cost(args, total * (blockIdx.x + 1) / gridDim.x);
+            if (ie > ib) { sm.chunk_item[0] = ib; sm.chunk_first[0] = 0; cnt = ie - ib; nch = 1; }
+        } else {
+            // Long sequences: every head is cut into `split` runs of equal cost, and the runs are dealt to the blocks
+            // in turn.  The blocks then work on gridDim.x / split heads at a time instead of one head each, so that
+            // the fp32 dQ accumulator lines of the heads in flight (and their Q, dO tiles) stay in L2.
+            const int n_runs = args.n_heads * args.split;
+            for (int k = blockIdx.x; k < n_runs && nch < MAX_CHUNKS; k += gridDim.x) {
+                const int head = k / args.split, c = k - head * args.split;
+                const int lo_cost = (int)((long long)args.head_cost * c / args.split);
+                const int hi_cost = (int)((long long)args.head_cost * (c + 1) / args.split);
+                const int tb = first_item_at_cost(args, lo_cost);                       // tile index: the head is 0 here
+                const int te = c + 1 == args.split ? n_work : first_item_at_cost(args, hi_cost);
+                if (te > tb) { sm.chunk_item[nch] = head * n_work + tb; sm.chunk_first[nch] = cnt; cnt += te - tb; ++nch; }
+            }
+        }
+        sm.chunk_first[nch] = cnt;
+        sm.n_chunks = nch;
     }
     for (int t = threadIdx.x; t < min(n_work, WORK_CACHE); t += NUM_THREADS) sm.work[t] = args.work[t];
     if (warp == MMA_WARP) {
@@ -262,7 +289,15 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
-    const int item_begin = sm.item_begin, item_end = sm.item_end;
+    const int n_chunks = sm.n_chunks, n_items = sm.chunk_first[n_chunks];
+    // item number n of this block (n rises, or steps back by one or two, from call to call: `run` follows it)
+    const int first_item = sm.chunk_item[0];
+    auto item_at = [&](int n, int& run) -> int {
+        if (!CHUNKED) return first_item + n;
+        while (n >= sm.chunk_first[run + 1] && run + 1 < n_chunks) ++run;
+        while (n < sm.chunk_first[run] && run > 0) --run;
+        return sm.chunk_item[run] + (n - sm.chunk_first[run]);
+    };
     volatile int* abort_flag = &sm.abort_flag;
 
     auto get_work = [&](int g) -> BwdWork {
@@ -291,11 +326,12 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
             bool ok = true;
             int gs = 0;                                     // steps issued so far, over all items
-            for (int g = item_begin; g < item_end && ok; ++g) {
+            int run = 0;
+            for (int item = 0; item < n_items && ok; ++item) {
+                const int g = item_at(item, run);
                 const int bh = g / n_work;
                 const BwdWork w = get_work(g);
                 const int n_steps = steps_of(w);
-                const int item = g - item_begin;
                 if (item >= 2) {
                     // the buffer held K of the item before the previous one, read by its dQ products
                     ok = __all_sync(0xffffffffu, mbar_wait(&sm.k_free[item & 1], ((item >> 1) & 1) ^ 1, abort_flag));
@@ -334,7 +370,9 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // their use (plain loads: their row offsets are not 16-byte aligned, so TMA cannot fetch them).
             bool ok = true;
             int gs = 0;
-            for (int g = item_begin; g < item_end && ok; ++g) {
+            int run = 0;
+            for (int item = 0; item < n_items && ok; ++item) {
+                const int g = item_at(item, run);
                 const int bh = g / n_work;
                 const BwdWork w = get_work(g);
                 const int n_steps = steps_of(w);
@@ -430,8 +468,9 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             // The steps of all items form one sequence: while the compute warpgroups work on a step, the
             // tensor core gets the next step's S^T, dP^T even when that step belongs to the next item (whose
             // K, V rows the drain warps have put into TMEM by then).
-            if (item_begin < item_end) {
-                const BwdWork w0 = get_work(item_begin);
+            int run = 0;
+            if (n_items > 0) {
+                const BwdWork w0 = get_work(item_at(0, run));
                 ok = wait2(&sm.kv_tmem, 0, &sm.qdo_full[0], 0, true, 0x1200);
                 if (ok) {
                     tc_fence_after();
@@ -439,17 +478,16 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         scores(0, half_cols(w0, 0, 0), 0);
                         const int n1 = half_cols(w0, 0, 1);
                         if (n1 > 0) scores(1, n1, 0);
-                        if (steps_of(w0) == 1 && item_begin + 1 < item_end) tc_commit(&sm.kv_free);
+                        if (steps_of(w0) == 1 && 1 < n_items) tc_commit(&sm.kv_free);
                     }
                     __syncwarp();
                 }
             }
-            for (int g = item_begin; g < item_end && ok; ++g) {
-                const BwdWork w = get_work(g);
+            for (int item = 0; item < n_items && ok; ++item) {
+                const BwdWork w = get_work(item_at(item, run));
                 const int n_steps = steps_of(w);
-                const int item = g - item_begin;
-                const bool next_item = g + 1 < item_end;
-                const BwdWork wn = next_item ? get_work(g + 1) : w;
+                const bool next_item = item + 1 < n_items;
+                const BwdWork wn = next_item ? get_work(item_at(item + 1, run)) : w;
                 const int n_steps_next = steps_of(wn);
                 const uint64_t k_mn = k_mn0 + (item & 1) * 1024;
                 for (int i = 0; i < n_steps && ok; ++i, ++gs) {
@@ -461,7 +499,7 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     const int m0 = more ? half_cols(w, i + 1, 0) : cross ? half_cols(wn, 0, 0) : 0;
                     const int m1 = more ? half_cols(w, i + 1, 1) : cross ? half_cols(wn, 0, 1) : 0;
                     // the next step is the last one that reads its item's K, V rows in TMEM, and another item follows
-                    const bool frees_kv = more ? (i + 2 == n_steps && next_item) : (cross && n_steps_next == 1 && g + 2 < item_end);
+                    const bool frees_kv = more ? (i + 2 == n_steps && next_item) : (cross && n_steps_next == 1 && item + 2 < n_items);
                     // ---- burst X: needs P^T, dS^T of half 0 and the next step's Q / dO tile
                     ok = wait2(&sm.p_full[0], ng[0] & 1, &sm.qdo_full[slot_next], ((gs + 1) / NSTAGE) & 1, any_next, 0x1400 + i);
                     if (!ok) break;
@@ -564,24 +602,25 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             mbar_arrive(&sm.kv_tmem);
             return true;
         };
-        if (item_begin < item_end) {
-            ok = copy_kv(item_begin, 0, false);
-            if (ok && steps_of(get_work(item_begin)) == 1 && item_begin + 1 < item_end) ok = copy_kv(item_begin + 1, 1, true);
+        int run = 0;
+        if (n_items > 0) {
+            ok = copy_kv(item_at(0, run), 0, false);
+            if (ok && steps_of(get_work(item_at(0, run))) == 1 && 1 < n_items) ok = copy_kv(item_at(1, run), 1, true);
         }
-        for (int g = item_begin; g < item_end && ok; ++g) {
+        for (int item = 0; item < n_items && ok; ++item) {
+            const int g = item_at(item, run);
             const int bh = g / n_work;
             const BwdWork w = get_work(g);
             const int n_steps = steps_of(w);
-            const int item = g - item_begin;
-            const bool next_item = g + 1 < item_end;
-            const int n_steps_next = next_item ? steps_of(get_work(g + 1)) : 0;
+            const bool next_item = item + 1 < n_items;
+            const int n_steps_next = next_item ? steps_of(get_work(item_at(item + 1, run))) : 0;
             for (int i = 0; i < n_steps; ++i, ++gs) {
                 const bool more = i + 1 < n_steps;
                 // the next step is the last one of its item and another item follows: that item's K, V rows
                 // go to TMEM as soon as the next step's scores are complete
-                if (more ? (i + 2 == n_steps && next_item) : (next_item && n_steps_next == 1 && g + 2 < item_end)) {
-                    const int gc = more ? g + 1 : g + 2;
-                    ok = copy_kv(gc, gc - item_begin, true);
+                if (more ? (i + 2 == n_steps && next_item) : (next_item && n_steps_next == 1 && item + 2 < n_items)) {
+                    const int nc = more ? item + 1 : item + 2;
+                    ok = copy_kv(item_at(nc, run), nc, true);
                     if (!ok) break;
                 }
                 if (!more) {
@@ -659,8 +698,9 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         int gs = 0;                                         // steps seen so far (aux ring, dS buffer parity)
         int nsh = 0;                                        // non-empty halves of this warpgroup seen so far
 
-        for (int g = item_begin; g < item_end && ok; ++g) {
-            const BwdWork w = get_work(g);
+        int run = 0;
+        for (int item = 0; item < n_items && ok; ++item) {
+            const BwdWork w = get_work(item_at(item, run));
             const int n_steps = steps_of(w);
             // the four key rows this thread works on in the softmax-gradient layout, and the queries that may see them
             const bool tile_masked = (!w.uniform) || (w.row_count < BKV);
@@ -796,7 +836,9 @@ cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUte
                           const CUtensorMap& dq_acc_map, const BwdArgs& args, const __nv_bfloat16* out, const __nv_bfloat16* dout,
                           __nv_bfloat16* dq, int BH, cudaStream_t stream) {
     const size_t smem = sizeof(SharedStorage) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(hmar_bwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const size_t n_rows = (size_t)BH * args.L;
     {
@@ -807,7 +849,19 @@ cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUte
         KernelTimer timer("hmar_bwd_tc_kernel", stream);
         const long long items = (long long)BH * args.n_work;
         const unsigned grid = (unsigned)(items < sm_count() ? items : sm_count());
-        hmar_bwd_tc_kernel<<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, args);
+        BwdArgs a = args;
+        // Long sequences only (measured: at L = 2240 the kernel does not care how many heads are in flight, at
+        // L = 9451 it is a fifth slower with one head per block): 8 runs per head, fewer if a block would get
+        // more runs than its table holds.
+        a.split = 0;
+        if (args.L >= 4096) {
+            a.split = 8;
+            while (a.split > 0 && ((long long)BH * a.split + grid - 1) / grid > MAX_CHUNKS) a.split >>= 1;
+        }
+        if (a.split > 0)
+            hmar_bwd_tc_kernel<true><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
+        else
+            hmar_bwd_tc_kernel<false><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
     }
     const size_t n8 = n_rows * D / 8;
     {

@@ -56,6 +56,7 @@ struct BwdArgs {
     int n_work;
     int n_heads;             // B * H
     int head_cost;           // from bwd_fill_costs
+    int split;               // set by the launcher: runs per head dealt to the blocks in turn (0: one contiguous run per block)
     int L;
     float scale_log2;        // softmax_scale * log2(e)
     float softmax_scale;
