@@ -32,7 +32,7 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
 # The captures are of the batch-4 case (traffic grows in proportion to the heads), scaled by 4 to the full batch.
-NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (235688704 + 118888192), "hmar_fwd": 4 * (82639872 + 10498816)}
+NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (231254016 + 111613440), "hmar_fwd": 4 * (82641152 + 11431936)}
 
 
 def pairs_per_head(side_lens):
