@@ -854,7 +854,7 @@ cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUte
         // L = 9451 it is a fifth slower with one head per block): 8 runs per head, fewer if a block would get
         // more runs than its table holds.
         a.split = 0;
-        if (args.L >= 4096) {
+        if (args.L >= 4096 && (unsigned)BH >= grid) {       // (with fewer heads than blocks the runs would not balance)
             a.split = 8;
             while (a.split > 0 && ((long long)BH * a.split + grid - 1) / grid > MAX_CHUNKS) a.split >>= 1;
         }
