@@ -411,13 +411,15 @@ def _finish(args, wl, world, rank, dev, total_ms, e2e_ms, fwd_ms, bwd_ms, launch
         dom_tf = f_bwd / (dom_ms * 1e-3) / 1e12
         cpu_base = None if args.no_cpu else time_oracle(wl, min(24, B * H), 2, 0)[0]
         elem = 2 * B * H * L * D
+        import paper_2506_04421_b200 as hmar
+        ws_bytes = hmar.hmar_attn_bwd_workspace_bytes(B, H, D, sides)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD + (f" (batch reduced to {B})" if args.batch > 0 else ""),
                        "B": B, "H": H, "L": L, "D": D, "side_lens": list(sides), "softmax_scale": scale, "passes": "fwd+bwd", "parallelism": f"replicas x{world}",
-                       "l2": "tensors larger than L2 (8 x 110 MB + 446 MB scratch per step), no flush"},
+                       "l2": f"tensors larger than L2 (8 x {elem / 1e6:.0f} MB + {ws_bytes / 1e6:.0f} MB workspace per step), no flush"},
             "fraction_of_peak": {"burst": value / world / peaks["bf16_tflops"],
                                  "sustained": value / world / (peaks["bf16_tflops_sustained"] or float("nan")),
                                  "nominal_2250": value / world / 2250.0, "peaks": peaks["source"]},

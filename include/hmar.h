@@ -98,7 +98,8 @@ size_t hmar_attn_bwd_workspace_bytes(int B, int H, int D, int n_scales, const in
  *   in : q, k, v, out, dout [B,H,L,D]; lse [B,H,L] as written by the forward.
  *   out: dq, dk, dv [B,H,L,D] (fully overwritten).
  *   workspace : device scratch of at least hmar_attn_bwd_workspace_bytes() bytes, 256-byte aligned.
- * dQ is accumulated with floating-point atomics, so its low-order bits may differ between runs. */
+ * dQ is accumulated in fp32 by bulk tensor reductions into global memory (cp.reduce.async.bulk.tensor),
+ * whose order is not fixed, so its low-order bits may differ between runs. */
 int hmar_attn_bwd(const void* q, const void* k, const void* v, const void* out, const float* lse,
                   const void* dout, void* dq, void* dk, void* dv,
                   void* workspace, size_t workspace_bytes,
@@ -129,12 +130,12 @@ int hmar_attn_bwd_window_f32(const float* q, const float* k, const float* v, con
  * device array inside the library image (about 8.6 MB, held by every GPU that loads the library until
  * the process exits).  It is meant for code that runs where cudaMalloc is off limits: under a framework
  * that owns all device memory through its own pool, inside a server plug-in that must not grow after
- * start-up, or wherever a call that may synchronise the device is forbidden.
- *   - Limit: B * H * L <= HMAR_NOALLOC_MAX_ROWS (and at most 512 work tiles per head); larger problems
- *     are rejected with HMAR_ERR_WORKSPACE before anything is launched.
- *   - The call itself never calls cudaMalloc, cudaFree or any allocating routine.  Its first call on a
- *     device looks up the array's device address (cudaGetSymbolAddress); make that first call outside
- *     any stream capture.
+ * start-up, or wherever cudaMalloc / cudaFree are forbidden because they may synchronise the device.
+ *   - Limit: B * H * L <= HMAR_NOALLOC_MAX_ROWS; larger problems are rejected with HMAR_ERR_WORKSPACE
+ *     before anything is launched.
+ *   - The call itself never calls cudaMalloc, cudaFree or any allocating routine, and copies nothing from
+ *     host memory: the work list travels as kernel parameters.  Its first call on a device looks up the
+ *     array's device address (cudaGetSymbolAddress); make that first call outside any stream capture.
  *   - All calls on a device share the array.  The array keeps whatever the previous call left in it;
  *     each call overwrites the work list and delta and clears the accumulator itself.  Two calls whose
  *     GPU work may overlap (different streams without an ordering between them) race on it: keep

@@ -76,8 +76,7 @@ def lib():
     L.hmar_status_string.argtypes = [i]
     L.hmar_status_string.restype = ctypes.c_char_p
     for name in EXPORTED_SYMBOLS:
-        if getattr(L, name).restype is ctypes.c_int:
-            pass
+        getattr(L, name)                     # a missing symbol fails here, at load time
     _LIB = L
     return L
 

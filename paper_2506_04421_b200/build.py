@@ -36,8 +36,7 @@ def build(force=False, verbose=False):
     if not force and not needs_build():
         return LIB_PATH
     cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else [])
-    cmd += os.environ.get("HMAR_NVCC_FLAGS", "").split()      # developer switches, e.g. -DHMAR_STAMPS
-    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB_PATH, "-lcuda"]
+    cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", LIB_PATH]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         sys.stderr.write(res.stdout + res.stderr)

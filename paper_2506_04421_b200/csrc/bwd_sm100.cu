@@ -60,12 +60,7 @@ constexpr int MAX_CHUNKS = 64;       // runs of consecutive items a block can be
 constexpr int NUM_COMPUTE_THREADS = 256;
 constexpr int DRAIN_WARP0 = 8, PRODUCER_WARP = 12, MMA_WARP = 13, AUX_WARP = 14;
 constexpr int NUM_THREADS = 512;
-#ifndef X_RC
-#define X_RC 160
-#define X_RD 88
-#define X_RM 104
-#endif
-constexpr int REGS_COMPUTE = X_RC, REGS_DRAIN = X_RD, REGS_MISC = X_RM;
+constexpr int REGS_COMPUTE = 160, REGS_DRAIN = 88, REGS_MISC = 104;
 static_assert(2 * REGS_COMPUTE + REGS_DRAIN + REGS_MISC == 4 * 128, "register budget of the block");
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t COL_ST = 0, COL_DPT = 128, COL_DK = 256, COL_DV = 320, COL_DQ = 384, COL_K = 448, COL_V = 480;

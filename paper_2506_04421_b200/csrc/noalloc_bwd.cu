@@ -15,6 +15,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <mutex>
 #include <vector>
 
@@ -26,8 +27,11 @@
 namespace hmar {
 
 constexpr size_t kMaxRows = HMAR_NOALLOC_MAX_ROWS;             // B * H * L
-constexpr size_t kMaxWork = 512;                               // backward work tiles of one head
-constexpr size_t kWorkBytes = kMaxWork * sizeof(BwdWork);      // 16 KB
+// Backward work tiles of one head: a scale of n rows gives at most n / 128 + 1 tiles and a packed tile ends at a
+// scale boundary, so a head has at most L / 128 + 2 * n_scales tiles; the size check below can therefore not be
+// passed by a list that does not fit here.
+constexpr size_t kMaxWork = kMaxRows / 128 + 2 * HMAR_MAX_SCALES;
+constexpr size_t kWorkBytes = kMaxWork * sizeof(BwdWork);      // 12 KB
 constexpr size_t kDeltaBytes = kMaxRows * sizeof(float);
 constexpr size_t kAccBytes = kMaxRows * kHeadDim * sizeof(float);
 constexpr size_t kScratchBytes = kWorkBytes + kDeltaBytes + kAccBytes;
@@ -49,6 +53,16 @@ static unsigned char* scratch_address() {
         addr[dev] = p;
     }
     return addr[dev];
+}
+
+// The work list reaches the scratch as kernel parameters: parameters are copied when the launch is enqueued,
+// so no host buffer has to outlive the call and no host-to-device copy (which, from pageable memory, may make
+// the host wait for the stream) is involved.
+constexpr int kFillChunk = 96;                                 // 96 x 32 bytes of parameters per launch
+struct WorkChunk { BwdWork w[kFillChunk]; };
+static __global__ void noalloc_fill_work_kernel(const WorkChunk chunk, int first, int count) {
+    BwdWork* dst = reinterpret_cast<BwdWork*>(g_noalloc_scratch);
+    for (int i = threadIdx.x; i < count; i += blockDim.x) dst[first + i] = chunk.w[i];
 }
 
 bool make_rows_map_bf16(CUtensorMap* map, const void* base, int heads, int rows);
@@ -79,7 +93,7 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
     ScaleTable st;
     build_scale_table(n_scales, side_lens, HMAR_WINDOW_MARKOV, &st);
     const std::vector<Tile> tiles = build_tiles(st, 1);
-    if (tiles.size() > kMaxWork) return HMAR_ERR_WORKSPACE;
+    if (tiles.size() > kMaxWork) return HMAR_ERR_WORKSPACE;     // cannot happen (see kMaxWork); kept as a guard
 
     int dev = 0, major = 0;
     if (cudaGetDevice(&dev) != cudaSuccess ||
@@ -91,7 +105,7 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
     unsigned char* scratch = scratch_address();
     if (scratch == nullptr) return HMAR_ERR_CUDA;
 
-    BwdWork host_work[kMaxWork];
+    static thread_local BwdWork host_work[kMaxWork];
     for (size_t i = 0; i < tiles.size(); ++i) {
         host_work[i] = BwdWork{};
         host_work[i].row_begin = tiles[i].row_begin;
@@ -102,11 +116,15 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
     }
     const int head_cost = bwd_fill_costs(host_work, (int)tiles.size());
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // Pageable source: the runtime stages it before returning, so the stack buffer may go away.
-    if (cudaMemcpyAsync(scratch, host_work, tiles.size() * sizeof(BwdWork), cudaMemcpyHostToDevice, s) != cudaSuccess) {
-        cudaGetLastError();
-        return HMAR_ERR_CUDA;
+    for (size_t first = 0; first < tiles.size(); first += kFillChunk) {
+        WorkChunk chunk;
+        const int count = (int)std::min<size_t>(kFillChunk, tiles.size() - first);
+        for (int i = 0; i < count; ++i) chunk.w[i] = host_work[first + i];
+        for (int i = count; i < kFillChunk; ++i) chunk.w[i] = BwdWork{};
+        noalloc_fill_work_kernel<<<1, 128, 0, s>>>(chunk, (int)first, count);
     }
+    if (cudaGetLastError() != cudaSuccess) return HMAR_ERR_CUDA;
+    count_launch((int)((tiles.size() + kFillChunk - 1) / kFillChunk));
 
     const int BH = B * H;
     CUtensorMap mq, mk, mv, mdo, macc;
