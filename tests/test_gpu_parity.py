@@ -240,8 +240,8 @@ def test_other_block_masks_fwd_bwd(sides, dtype, window):
 
 def _sample_heads(BH, n=6):
     rng = np.random.default_rng(BH)
-    picks = {0, BH - 1} | set(int(x) for x in rng.integers(0, BH, size=n))
-    return sorted(picks)
+    inner = rng.permutation(np.arange(1, BH - 1))[:max(0, min(n, BH) - 2)]
+    return sorted({0, BH - 1} | set(int(x) for x in inner))
 
 
 def _partition_heads(wl, n, window=hmar.HMAR_WINDOW_MARKOV):
