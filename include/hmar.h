@@ -154,7 +154,9 @@ int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v, const voi
  *                                     must be NULL iff side_prev == 0 (first scale)
  *   k_cur, v_cur : [B,H,n_cur,D]      the current scale's own keys / values
  *   out          : [B,H,n_cur,D];  lse : [B,H,n_cur] fp32 or NULL.
- * Dense attention of q over (prev followed by cur); no mask inside the window. */
+ * Dense attention of q over (prev followed by cur); no mask inside the window.
+ * Windows of at most 128 keys (and 96 queries) run in a kernel of their own: one block per head, K and V
+ * of the head in shared memory, warp-level bf16 products; larger ones in the forward kernel's two-segment mode. */
 int hmar_attn_scale_step(const void* q, const void* k_prev, const void* v_prev,
                          const void* k_cur, const void* v_cur, void* out, float* lse,
                          int B, int H, int D, int side_prev, int side_cur,
@@ -163,6 +165,20 @@ int hmar_attn_scale_step_f32(const float* q, const float* k_prev, const float* v
                              const float* k_cur, const float* v_cur, float* out, float* lse,
                              int B, int H, int D, int side_prev, int side_cur,
                              float softmax_scale, void* stream);
+/* The same step on tensors whose heads are not packed back to back (Sec. 1 / Sec. 5.2: inference keeps only
+ * the previous scale's keys and values, so a sampler holds them in one small ring and must not copy them
+ * to concatenate).  Rows are D contiguous elements; head b*H + h of a tensor starts `*_head_stride`
+ * elements after head b*H + h - 1 (each at least rows * D and a multiple of 8).  With K and V of the
+ * previous and the current scale adjacent in one buffer [B,H,ring_rows,D]: k_cur = k_prev + n_prev * D
+ * and kv_prev_head_stride = kv_cur_head_stride = ring_rows * D.  bf16 only; lse stays [B,H,n_cur] dense.
+ * Errors as hmar_attn_scale_step; with the plain-kernel debug switch on, only dense strides are accepted
+ * (HMAR_ERR_UNSUPPORTED otherwise). */
+int hmar_attn_scale_step_strided(const void* q, const void* k_prev, const void* v_prev,
+                                 const void* k_cur, const void* v_cur, void* out, float* lse,
+                                 int B, int H, int D, int side_prev, int side_cur,
+                                 long long q_head_stride, long long kv_prev_head_stride,
+                                 long long kv_cur_head_stride, long long out_head_stride,
+                                 float softmax_scale, void* stream);
 
 /* Host-side scale-block scheduler (Sec. 4.1: the kernel visits only the live blocks of the mask).
  * Writes the work list of one head for `direction` 0 = forward (tiles of query rows, each with the

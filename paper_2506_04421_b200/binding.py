@@ -28,7 +28,7 @@ HMAR_WINDOW_SELF = 2        # scale k only (block-diagonal)
 EXPORTED_SYMBOLS = (
     "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_fwd_window", "hmar_attn_fwd_window_f32", "hmar_attn_fwd_packed",
     "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd", "hmar_attn_bwd_f32", "hmar_attn_bwd_window",
-    "hmar_attn_bwd_window_f32", "hmar_schedule_tiles_window", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_schedule_tiles",
+    "hmar_attn_bwd_window_f32", "hmar_schedule_tiles_window", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_attn_scale_step_strided", "hmar_schedule_tiles",
     "hmar_device_status", "hmar_profile_begin", "hmar_profile_end", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
     "hmar_status_string",
 )
@@ -66,6 +66,8 @@ def lib():
     L.hmar_attn_bwd_noalloc.argtypes = [vp] * 9 + [i, i, i, i, ip, fp, vp]
     L.hmar_attn_scale_step.argtypes = [vp] * 7 + [i, i, i, i, i, fp, vp]
     L.hmar_attn_scale_step_f32.argtypes = L.hmar_attn_scale_step.argtypes
+    ll = ctypes.c_longlong
+    L.hmar_attn_scale_step_strided.argtypes = [vp] * 7 + [i, i, i, i, i, ll, ll, ll, ll, fp, vp]
     L.hmar_schedule_tiles.argtypes = [i, ip, i, ctypes.POINTER(ctypes.c_int32), i]
     L.hmar_device_status.argtypes = [ip]
     L.hmar_profile_begin.restype = None
@@ -221,6 +223,33 @@ def hmar_attn_scale_step(q, k_prev, v_prev, k_cur, v_cur, side_prev, side_cur, s
     _check(fn(_ptr(q), _ptr(k_prev), _ptr(v_prev), _ptr(k_cur), _ptr(v_cur), _ptr(out), _ptr(lse),
               B, H, D, int(side_prev), int(side_cur), float(softmax_scale), _stream(stream)),
            "hmar_attn_scale_step")
+    return out, lse
+
+
+def hmar_attn_scale_step_strided(q, k_prev, v_prev, k_cur, v_cur, side_prev, side_cur, softmax_scale,
+                                 out=None, lse=None, want_lse=True, stream=None):
+    """Inference step on views whose heads are not packed back to back, e.g. slices of one K/V ring
+    [B,H,ring_rows,D] (k_prev = ring[:, :, a:a+n_prev], k_cur = ring[:, :, a+n_prev:a+n_prev+n_cur]).
+    Every tensor is a [B,H,rows,D] view with contiguous rows and heads a constant stride apart."""
+    B, H, n_cur, D = q.shape
+
+    def head_stride(t):
+        if t is None:
+            return 0
+        if not t.is_cuda or t.stride(3) != 1 or t.stride(2) != D or (t.shape[1] > 1 and t.shape[0] > 1 and t.stride(0) != H * t.stride(1)):
+            raise ValueError("views must have contiguous rows and evenly spaced heads")
+        return t.stride(1) if t.shape[1] > 1 else (t.stride(0) if t.shape[0] > 1 else t.shape[2] * D)
+
+    if _is_f32(q):
+        raise TypeError("hmar_attn_scale_step_strided takes bfloat16 tensors")
+    if out is None:
+        out = torch.empty((B, H, n_cur, D), dtype=q.dtype, device=q.device)
+    if lse is None and want_lse:
+        lse = torch.empty((B, H, n_cur), dtype=torch.float32, device=q.device)
+    _check(lib().hmar_attn_scale_step_strided(
+        _ptr(q), _ptr(k_prev), _ptr(v_prev), _ptr(k_cur), _ptr(v_cur), _ptr(out), _ptr(lse), B, H, D, int(side_prev),
+        int(side_cur), head_stride(q), head_stride(k_prev), head_stride(k_cur), head_stride(out), float(softmax_scale),
+        _stream(stream)), "hmar_attn_scale_step_strided")
     return out, lse
 
 

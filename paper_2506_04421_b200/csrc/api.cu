@@ -162,10 +162,11 @@ static int bwd_impl(const T* q, const T* k, const T* v, const T* out, const floa
                ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
+// strides == nullptr: dense [B,H,n,D] tensors
 template <typename T>
 static int step_impl(const T* q, const T* k_prev, const T* v_prev, const T* k_cur, const T* v_cur, T* out,
-                     float* lse, int B, int H, int D, int side_prev, int side_cur, float softmax_scale,
-                     void* stream, bool tensor_core) {
+                     float* lse, int B, int H, int D, int side_prev, int side_cur, const StepStrides* strides,
+                     float softmax_scale, void* stream, bool tensor_core) {
     int rc = check_shape(B, H, D);
     if (rc != HMAR_OK) return rc;
     if (side_cur <= 0 || side_cur > 4096 || side_prev < 0 || side_prev > 4096) return HMAR_ERR_BAD_ARG;
@@ -176,15 +177,28 @@ static int step_impl(const T* q, const T* k_prev, const T* v_prev, const T* k_cu
     const void* ptrs[] = {q, k_prev, v_prev, k_cur, v_cur, out, lse};
     for (const void* p : ptrs)
         if (!aligned16(p)) return HMAR_ERR_BAD_ARG;
+    const int n_prev = side_prev * side_prev, n_cur = side_cur * side_cur;
+    StepStrides st{(long long)n_cur * D, (long long)n_prev * D, (long long)n_cur * D, (long long)n_cur * D};
+    bool dense = true;
+    if (strides != nullptr) {
+        // a head must hold its rows, and heads must start on 16-byte boundaries
+        if (strides->q < st.q || strides->kv_cur < st.kv_cur || strides->out < st.out ||
+            (n_prev > 0 && strides->kv_prev < st.kv_prev))
+            return HMAR_ERR_BAD_ARG;
+        if (((strides->q | strides->kv_prev | strides->kv_cur | strides->out) & 7) != 0) return HMAR_ERR_BAD_ARG;
+        dense = strides->q == st.q && strides->kv_cur == st.kv_cur && strides->out == st.out &&
+                (n_prev == 0 || strides->kv_prev == st.kv_prev);
+        st = *strides;
+    }
     rc = check_device();
     if (rc != HMAR_OK) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const int n_prev = side_prev * side_prev, n_cur = side_cur * side_cur;
     if constexpr (std::is_same<T, __nv_bfloat16>::value) {
         if (tensor_core && !g_force_simt.load())
-            return tc_scale_step(q, k_prev, v_prev, k_cur, v_cur, out, lse, B * H, n_prev, n_cur, softmax_scale,
+            return tc_scale_step(q, k_prev, v_prev, k_cur, v_cur, out, lse, B * H, n_prev, n_cur, st, softmax_scale,
                                  device_status_ptr(), s);
     }
+    if (!dense) return HMAR_ERR_UNSUPPORTED;      // the plain kernels take dense tensors only
     return simt_scale_step<T>(q, k_prev, v_prev, k_cur, v_cur, out, lse, B * H, n_prev, n_cur, softmax_scale, s)
                    == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
@@ -277,14 +291,25 @@ int hmar_attn_scale_step(const void* q, const void* k_prev, const void* v_prev, 
                          const void* v_cur, void* out, float* lse, int B, int H, int D, int side_prev,
                          int side_cur, float softmax_scale, void* stream) {
     return step_impl<bf16>((const bf16*)q, (const bf16*)k_prev, (const bf16*)v_prev, (const bf16*)k_cur,
-                           (const bf16*)v_cur, (bf16*)out, lse, B, H, D, side_prev, side_cur, softmax_scale,
+                           (const bf16*)v_cur, (bf16*)out, lse, B, H, D, side_prev, side_cur, nullptr, softmax_scale,
+                           stream, true);
+}
+
+int hmar_attn_scale_step_strided(const void* q, const void* k_prev, const void* v_prev, const void* k_cur,
+                                 const void* v_cur, void* out, float* lse, int B, int H, int D, int side_prev,
+                                 int side_cur, long long q_head_stride, long long kv_prev_head_stride,
+                                 long long kv_cur_head_stride, long long out_head_stride, float softmax_scale,
+                                 void* stream) {
+    const StepStrides st{q_head_stride, kv_prev_head_stride, kv_cur_head_stride, out_head_stride};
+    return step_impl<bf16>((const bf16*)q, (const bf16*)k_prev, (const bf16*)v_prev, (const bf16*)k_cur,
+                           (const bf16*)v_cur, (bf16*)out, lse, B, H, D, side_prev, side_cur, &st, softmax_scale,
                            stream, true);
 }
 
 int hmar_attn_scale_step_f32(const float* q, const float* k_prev, const float* v_prev, const float* k_cur,
                              const float* v_cur, float* out, float* lse, int B, int H, int D, int side_prev,
                              int side_cur, float softmax_scale, void* stream) {
-    return step_impl<float>(q, k_prev, v_prev, k_cur, v_cur, out, lse, B, H, D, side_prev, side_cur,
+    return step_impl<float>(q, k_prev, v_prev, k_cur, v_cur, out, lse, B, H, D, side_prev, side_cur, nullptr,
                             softmax_scale, stream, false);
 }
 

@@ -214,15 +214,19 @@ int tc_fwd_packed(const bf16* qkv, bf16* out, float* lse, int B, int H, const Sc
 }
 
 int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const bf16* k_cur, const bf16* v_cur,
-                  bf16* out, float* lse, int BH, int n_prev, int n_cur, float scale, int* status,
+                  bf16* out, float* lse, int BH, int n_prev, int n_cur, const StepStrides& st, float scale, int* status,
                   cudaStream_t stream) {
+    if (step_small_applies(n_prev, n_cur))
+        return step_small(q, k_prev, v_prev, k_cur, v_cur, out, lse, BH, n_prev, n_cur, st.q, st.kv_prev, st.kv_cur, st.out,
+                          scale, stream);
     CUtensorMap mq, mk0, mv0, mk1, mv1;
-    auto rows_map = [&](CUtensorMap* m, const bf16* base, int rows) {
-        return make_rows_map4(m, base, 1, BH, rows, kHeadDim, (long long)rows * kHeadDim, (long long)BH * rows * kHeadDim);
+    auto rows_map = [&](CUtensorMap* m, const bf16* base, int rows, long long head_stride) {
+        return make_rows_map4(m, base, 1, BH, rows, kHeadDim, head_stride, (long long)BH * head_stride);
     };
-    if (!rows_map(&mq, q, n_cur) || !rows_map(&mk1, k_cur, n_cur) || !rows_map(&mv1, v_cur, n_cur)) return HMAR_ERR_CUDA;
+    if (!rows_map(&mq, q, n_cur, st.q) || !rows_map(&mk1, k_cur, n_cur, st.kv_cur) || !rows_map(&mv1, v_cur, n_cur, st.kv_cur))
+        return HMAR_ERR_CUDA;
     if (n_prev > 0) {
-        if (!rows_map(&mk0, k_prev, n_prev) || !rows_map(&mv0, v_prev, n_prev)) return HMAR_ERR_CUDA;
+        if (!rows_map(&mk0, k_prev, n_prev, st.kv_prev) || !rows_map(&mv0, v_prev, n_prev, st.kv_prev)) return HMAR_ERR_CUDA;
     } else {
         mk0 = mk1;
         mv0 = mv1;
@@ -233,8 +237,8 @@ int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const b
     a.n_q_rows = n_cur;
     a.heads_per_batch = BH;
     a.out_row_stride = kHeadDim;
-    a.out_head_stride = (long long)n_cur * kHeadDim;
-    a.out_batch_stride = (long long)BH * n_cur * kHeadDim;
+    a.out_head_stride = st.out;
+    a.out_batch_stride = (long long)BH * st.out;
     a.n0 = n_prev;
     a.n1 = n_cur;
     a.scale_log2 = scale * 1.4426950408889634f;

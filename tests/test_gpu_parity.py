@@ -341,15 +341,17 @@ def test_scale_step_small_batch_all_scales(dtype):
     _no_device_error()
 
 
-def test_scale_step_full_batch_last_scales_sampled_heads():
-    """Config 5 at B=64, H=24 for the three largest scales; sampled heads against the oracle."""
+@pytest.mark.parametrize("sub", [0, 3])
+def test_scale_step_full_batch_all_scales_sampled_heads(sub):
+    """Config 5 at B=64, H=24, every scale, first and last masked sub-step; sampled heads against the oracle.
+    Scales 1-6 (windows of at most 128 keys) run in the small-window kernel, 7-10 in the tcgen05 kernel."""
     wl = CONFIGS["512_d24_infer"]
     BH = wl.B * wl.H
-    heads = _sample_heads(BH, 2)
+    heads = _sample_heads(BH, 6)
     idx = torch.as_tensor(heads, device="cuda")
-    for s in (0, 7, 8, 9):
+    for s in range(len(wl.side_lens)):
         side, side_prev = wl.side_lens[s], (wl.side_lens[s - 1] if s else 0)
-        host = scale_step_inputs(wl, s, 1, bf16=True, heads=heads)
+        host = scale_step_inputs(wl, s, sub, bf16=True, heads=heads)
         dev = []
         for sid, h in enumerate(host):
             if h is None:
@@ -362,8 +364,52 @@ def test_scale_step_full_batch_last_scales_sampled_heads():
         ref_out, ref_lse = orc.scale_step(*host, wl.softmax_scale)
         _assert_close(f"out[scale {s}]", out.view(BH, -1, wl.D)[idx], ref_out, False)
         _assert_lse(lse.view(BH, -1)[idx], ref_lse, False)
-        assert torch.isfinite(out).all()
+        assert torch.isfinite(out).all() and torch.isfinite(lse).all()
     _no_device_error()
+
+
+@pytest.mark.parametrize("sides", [(1, 2), (3, 4, 6), (9, 13), (13, 18), (18, 24), (5, 14)])
+def test_scale_step_on_a_kv_ring_matches_dense_tensors_bits(sides):
+    """K and V of the previous and the current scale adjacent in one ring buffer [B,H,ring_rows,D], q and out
+    as slices of wider buffers: the strided entry point must give the oracle's result and the very bits of
+    the dense entry point (both kernels: windows below and above 128 keys)."""
+    wl = _Wl(sides, B=2, H=3)
+    B, H, D = wl.B, wl.H, wl.D
+    for s in range(1, len(sides)):
+        n_prev, n_cur = sides[s - 1] ** 2, sides[s] ** 2
+        q, kp, vp, kc, vc = scale_step_inputs(wl, s, 0, bf16=True)
+        ring_rows = n_prev + n_cur + 24
+        ring_k = torch.full((B, H, ring_rows, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+        ring_v = torch.full_like(ring_k, float("nan"))
+        a = 8
+        for ring, prev, cur in ((ring_k, kp, kc), (ring_v, vp, vc)):
+            ring[:, :, a:a + n_prev] = to_device(prev, B, H, torch.bfloat16)
+            ring[:, :, a + n_prev:a + n_prev + n_cur] = to_device(cur, B, H, torch.bfloat16)
+        q_wide = torch.zeros((B, H, n_cur + 8, D), dtype=torch.bfloat16, device="cuda")
+        q_wide[:, :, :n_cur] = to_device(q, B, H, torch.bfloat16)
+        out_wide = torch.full((B, H, n_cur + 16, D), 7.0, dtype=torch.bfloat16, device="cuda")
+        out, lse = hmar.hmar_attn_scale_step_strided(
+            q_wide[:, :, :n_cur], ring_k[:, :, a:a + n_prev], ring_v[:, :, a:a + n_prev],
+            ring_k[:, :, a + n_prev:a + n_prev + n_cur], ring_v[:, :, a + n_prev:a + n_prev + n_cur],
+            sides[s - 1], sides[s], wl.softmax_scale, out=out_wide[:, :, :n_cur])
+        ref_out, ref_lse = orc.scale_step(q, kp, vp, kc, vc, wl.softmax_scale)
+        _assert_close("out", out_wide[:, :, :n_cur].contiguous(), ref_out, False)
+        _assert_lse(lse, ref_lse, False)
+        assert (out_wide[:, :, n_cur:] == 7.0).all()                     # nothing written past the head's rows
+        dense = [to_device(x, B, H, torch.bfloat16) for x in (q, kp, vp, kc, vc)]
+        out_d, lse_d = hmar.hmar_attn_scale_step(*dense, sides[s - 1], sides[s], wl.softmax_scale)
+        assert torch.equal(out_d, out_wide[:, :, :n_cur]) and torch.equal(lse_d, lse)
+    _no_device_error()
+
+
+def test_scale_step_strided_argument_errors():
+    import ctypes
+    p = ctypes.c_void_p(1 << 12)
+    f = hmar.lib().hmar_attn_scale_step_strided
+    ok_strides = (16 * 64, 4 * 64, 16 * 64, 16 * 64)
+    assert f(p, p, p, p, p, p, None, 1, 1, 64, 2, 4, 16 * 64 - 8, *ok_strides[1:], 0.125, None) == hmar.HMAR_ERR_BAD_ARG   # head shorter than its rows
+    assert f(p, p, p, p, p, p, None, 1, 1, 64, 2, 4, 16 * 64 + 4, *ok_strides[1:], 0.125, None) == hmar.HMAR_ERR_BAD_ARG   # heads off the 16-byte grid
+    assert f(p, None, None, p, p, p, None, 1, 1, 64, 2, 4, *ok_strides, 0.125, None) == hmar.HMAR_ERR_BAD_ARG              # prev missing
 
 
 def test_full_size_forward_and_scale_step_repeat_bit_identical():
