@@ -153,27 +153,153 @@ def time_dense_masked(wl, q, k, v, do, reps=3):
     return e0.elapsed_time(e1) / reps
 
 
-def time_scale_steps(hmar, wl_inf, dev, reps=5):
-    """ms per inference step of every scale of the 512x512 d24 inference sweep (B=64, H=24; each step is
-    one masked sub-step: fresh Q and own-scale K/V, the previous scale's K/V kept)."""
+L2_BYTES = 126 * 1024 * 1024
+
+
+def _rotating_sets(bytes_per_set, cap=12):
+    """How many copies of a leg's tensors to cycle through so that consecutive iterations do not find their
+    inputs in L2 (the sets together hold more than twice the L2, up to `cap` sets)."""
+    return int(max(2, min(cap, -(-2 * L2_BYTES // max(1, bytes_per_set)))))
+
+
+def time_scale_steps(hmar, wl_inf, dev, peaks, reps=6):
+    """Every scale of the 512x512 d24 inference sweep (B=64, H=24; one call is one masked sub-step: fresh Q and
+    own-scale K/V, the previous scale's K/V kept).  Per scale: ms per call (CUDA events around `reps` calls that
+    cycle through several input sets, so the inputs come from HBM), achieved GB/s on the algorithmic bytes
+    (Q, O, K/V of both scales once) and useful TFLOP/s, each as a fraction of its measured peak."""
     import torch
     from workloads.device import bulk_normal
-    out = []
+    B, H, D = wl_inf.B, wl_inf.H, wl_inf.D
+    rows = []
     for s, side in enumerate(wl_inf.side_lens):
         side_prev = wl_inf.side_lens[s - 1] if s else 0
-        t = [bulk_normal(wl_inf.seed + s, i, wl_inf.B, wl_inf.H, (side_prev if i in (1, 2) else side) ** 2, wl_inf.D,
-                         torch.bfloat16, dev) if (s or i not in (1, 2)) else None for i in range(5)]
-        o = torch.empty_like(t[0])
-        for _ in range(2):
-            hmar.hmar_attn_scale_step(*t, side_prev, side, wl_inf.softmax_scale, out=o, want_lse=False)
+        nc, npv = side * side, side_prev * side_prev
+        byt = B * H * (2 * nc + 2 * (nc + npv)) * D * 2
+        flops = 4 * B * H * nc * (nc + npv) * D
+        n_sets = _rotating_sets(byt)
+        sets = []
+        for k in range(n_sets):
+            sets.append([bulk_normal(wl_inf.seed + s + 100 * k, i, B, H, (side_prev if i in (1, 2) else side) ** 2, D,
+                                     torch.bfloat16, dev) if (s or i not in (1, 2)) else None for i in range(5)])
+        o = torch.empty_like(sets[0][0])
+        for k in range(min(3, n_sets)):
+            hmar.hmar_attn_scale_step(*sets[k], side_prev, side, wl_inf.softmax_scale, out=o, want_lse=False)
+        n_calls = reps * n_sets if byt < (8 << 20) else max(reps, n_sets)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for _ in range(reps):
-            hmar.hmar_attn_scale_step(*t, side_prev, side, wl_inf.softmax_scale, out=o, want_lse=False)
+        for it in range(n_calls):
+            hmar.hmar_attn_scale_step(*sets[it % n_sets], side_prev, side, wl_inf.softmax_scale, out=o, want_lse=False)
         e1.record()
         torch.cuda.synchronize()
-        out.append(round(e0.elapsed_time(e1) / reps, 4))
-    return out
+        ms = e0.elapsed_time(e1) / n_calls
+        gbs, tf = byt / ms / 1e6, flops / ms / 1e9
+        rows.append({"scale": s + 1, "side": side, "ms": round(ms, 4), "gbs": round(gbs, 1),
+                     "frac_hbm": round(gbs / peaks["hbm_gbs"], 4), "tflops": round(tf, 1),
+                     "frac_tensor": round(tf / peaks["bf16_tflops"], 4), "input_sets": n_sets,
+                     "bound": "tensor" if flops / byt > 250 else ("hbm" if byt > (16 << 20) else "launch latency")})
+        del sets
+        torch.cuda.empty_cache()
+    return rows
+
+
+def time_small_config(hmar, wl_x, dev, peaks, reps=4):
+    """A 256x256 (L = 680) config at its full batch: forward, and backward if the config has one.  The tensors of
+    these configs fit in L2, so the calls cycle through several input sets.  Reports ms, useful TFLOP/s, and GB/s
+    on the algorithmic bytes (fwd: Q, K, V, O + LSE; bwd: Q, K, V, O, dO, LSE in, dQ, dK, dV out) against the
+    measured HBM copy bandwidth: these shapes are HBM-bound (arithmetic intensity 130-150 FLOP/B)."""
+    import torch
+    from workloads.device import bulk_normal
+    B, H, L, D = wl_x.B, wl_x.H, wl_x.L, wl_x.D
+    backward = "bwd" in wl_x.passes
+    elem = B * H * L * D * 2
+    fwd_bytes = 4 * elem + 4 * B * H * L
+    bwd_bytes = 8 * elem + 4 * B * H * L
+    n_sets = _rotating_sets(fwd_bytes + (bwd_bytes if backward else 0), cap=8)
+    sets = [[bulk_normal(wl_x.seed + 100 * k, i, B, H, L, D, torch.bfloat16, dev) for i in range(4 if backward else 3)]
+            for k in range(n_sets)]
+    out = torch.empty_like(sets[0][0])
+    lse = torch.empty((B, H, L), dtype=torch.float32, device=dev)
+    dq, dk, dv = (torch.empty_like(out) for _ in range(3)) if backward else (None, None, None)
+    ws = torch.empty(hmar.hmar_attn_bwd_workspace_bytes(B, H, D, wl_x.side_lens), dtype=torch.uint8, device=dev) if backward else None
+
+    def one(t):
+        hmar.hmar_attn_fwd(t[0], t[1], t[2], wl_x.side_lens, wl_x.softmax_scale, out=out, lse=lse)
+        if backward:
+            hmar.hmar_attn_bwd(t[0], t[1], t[2], out, lse, t[3], wl_x.side_lens, wl_x.softmax_scale, dq=dq, dk=dk, dv=dv,
+                               workspace=ws)
+
+    for t in sets[:2]:
+        one(t)
+    torch.cuda.synchronize()
+    n_calls = reps * n_sets
+    hmar.hmar_profile_begin()
+    for it in range(n_calls):
+        one(sets[it % n_sets])
+    kern = hmar.hmar_profile_end()
+    f_ms = kern["hmar_fwd_tc_kernel"][1] / n_calls
+    f_fl, b_fl = useful_flops(wl_x)
+    res = {"B": B, "H": H, "L": L, "input_sets": n_sets,
+           "fwd": {"ms": round(f_ms, 4), "tflops": round(f_fl / f_ms / 1e9, 1), "gbs": round(fwd_bytes / f_ms / 1e6, 1),
+                   "frac_hbm": round(fwd_bytes / f_ms / 1e6 / peaks["hbm_gbs"], 4), "algorithmic_bytes": fwd_bytes}}
+    if backward:
+        b_ms = sum(v[1] for k, v in kern.items() if "bwd" in k) / n_calls
+        res["bwd"] = {"ms": round(b_ms, 4), "tflops": round(b_fl / b_ms / 1e9, 1), "gbs": round(bwd_bytes / b_ms / 1e6, 1),
+                      "frac_hbm": round(bwd_bytes / b_ms / 1e6 / peaks["hbm_gbs"], 4), "algorithmic_bytes": bwd_bytes,
+                      "kernels_ms": {k: round(v[1] / n_calls, 4) for k, v in kern.items() if "bwd" in k}}
+    res["timing"] = "sum of the library's per-kernel CUDA events over the calls"
+    return res
+
+
+def oracle_errors(hmar, dev):
+    """Max / mean abs error against the CPU oracle of one head per config, the head placed in an otherwise
+    device-generated full-size problem (outside every timed region)."""
+    import torch
+    from oracle import hmar_oracle as orc
+    from workloads import CONFIGS, scale_step_inputs
+    from workloads.device import bulk_normal, training_tensors
+    res = {}
+
+    def err(g, r):
+        d = np.abs(g.detach().double().cpu().numpy().reshape(r.shape) - r)
+        return [float(f"{d.max():.3e}"), float(f"{d.mean():.3e}")]
+
+    for name in ("256_d16_fwd", "256_d30_train", "512_d24_train"):
+        wl_x = CONFIGS[name]
+        head = (wl_x.B * wl_x.H) // 3
+        backward = "bwd" in wl_x.passes
+        d, h = training_tensors(wl_x, [head], with_dout=backward)
+        out, lse = hmar.hmar_attn_fwd(d["q"], d["k"], d["v"], wl_x.side_lens, wl_x.softmax_scale)
+        ro, rl = orc.attn_fwd(h["q"], h["k"], h["v"], wl_x.side_lens, wl_x.softmax_scale)
+        e = {"head": head, "out": err(out.view(-1, wl_x.L, wl_x.D)[head], ro[0]), "lse": err(lse.view(-1, wl_x.L)[head], rl[0])}
+        if backward:
+            g = hmar.hmar_attn_bwd(d["q"], d["k"], d["v"], out, lse, d["dout"], wl_x.side_lens, wl_x.softmax_scale)
+            r = orc.attn_bwd(h["q"], h["k"], h["v"], h["dout"], wl_x.side_lens, wl_x.softmax_scale)
+            for nm, gg, rr in zip(("dq", "dk", "dv"), g, r):
+                e[nm] = err(gg.view(-1, wl_x.L, wl_x.D)[head], rr[0])
+        res[name] = e
+        del d
+        torch.cuda.empty_cache()
+    wl_i = CONFIGS["512_d24_infer"]
+    BH, head = wl_i.B * wl_i.H, (wl_i.B * wl_i.H) // 3
+    worst = [0.0, 0.0]
+    for s_, side in enumerate(wl_i.side_lens):
+        sp = wl_i.side_lens[s_ - 1] if s_ else 0
+        host = scale_step_inputs(wl_i, s_, 1, bf16=True, heads=[head])
+        devt = []
+        for sid, hh in enumerate(host):
+            if hh is None:
+                devt.append(None)
+                continue
+            t = bulk_normal(wl_i.seed + s_, sid, wl_i.B, wl_i.H, hh.shape[1], wl_i.D)
+            t.view(BH, hh.shape[1], wl_i.D)[head] = torch.from_numpy(hh[0]).to(device=dev, dtype=torch.bfloat16)
+            devt.append(t)
+        o, _ = hmar.hmar_attn_scale_step(*devt, sp, side, wl_i.softmax_scale)
+        ro, _ = orc.scale_step(*host, wl_i.softmax_scale)
+        e = err(o.view(BH, -1, wl_i.D)[head], ro[0])
+        worst = [max(worst[0], e[0]), max(worst[1], e[1])]
+    res["512_d24_infer"] = {"head": head, "out_worst_scale": worst}
+    res["what"] = "[max abs, mean abs] against the fp64 oracle, one head per config"
+    return res
 
 
 def time_training_shape(hmar, wl_x, dev, window, reps=3):
@@ -328,9 +454,21 @@ def run_ours(args, wl):
         torch.cuda.empty_cache()
         if args.batch == 0:
             from workloads import CONFIGS
-            ms = time_scale_steps(hmar, CONFIGS["512_d24_infer"], dev)
+            peaks = measured_peaks()
+            rows = time_scale_steps(hmar, CONFIGS["512_d24_infer"], dev, peaks)
+            ms = [r["ms"] for r in rows]
             extras["scale_step_ms"] = {"workload": "512_d24_infer, B=64 H=24, one sub-step per call", "per_scale": ms,
-                                       "sweep_4_sub_steps": round(4 * sum(ms), 4)}
+                                       "sweep_4_sub_steps": round(4 * sum(ms), 4), "roofline_per_scale": rows,
+                                       "peaks": {"hbm_gbs": peaks["hbm_gbs"], "bf16_tflops": peaks["bf16_tflops"], "source": peaks["source"]}}
+            torch.cuda.empty_cache()
+            # the two 256 x 256 configs (L = 680): HBM-bound shapes, achieved GB/s against the measured copy bandwidth
+            for nm in ("256_d16_fwd", "256_d30_train"):
+                extras[nm] = time_small_config(hmar, CONFIGS[nm], dev, peaks)
+                torch.cuda.empty_cache()
+            try:
+                extras["oracle_errors"] = oracle_errors(hmar, dev)
+            except Exception as e:     # context; its failure must not lose the benchmark line
+                extras["oracle_errors"] = {"error": str(e)[:200]}
             torch.cuda.empty_cache()
             # VAR's block-causal mask on the same shape and kernels: the workload the paper's speedups are against
             cf, cb = time_training_shape(hmar, wl, dev, hmar.HMAR_WINDOW_CAUSAL)
