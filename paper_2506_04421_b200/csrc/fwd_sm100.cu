@@ -3,27 +3,27 @@
 // One block handles one work tile: up to 128 consecutive query rows of one head and the contiguous
 // key range those rows may see under the mask (paper Sec. 4.1, Fig. attn-mask).  It is the usual
 // IO-aware tiling with an online softmax (Sec. 4.1: the kernel extends FlashAttention), laid out for
-// Blackwell.  Every 128-key tile is split into two halves of 64 keys, and each half has its own softmax
-// warpgroup, its own running maximum and row sum, and its own output accumulator: the two halves are
-// two independent attention problems over disjoint key sets, merged exactly at the end
-// (O = (w_a O_a + w_b O_b) / (w_a l_a + w_b l_b), w_x = 2^(m_x - max(m_a, m_b))).  Nothing ties the two
-// chains together, so one waits for the tensor core while the other computes, and two blocks per SM
-// give four such chains.
-//   warps 0-3   softmax of half a: one query row per thread, 64 logits per tile read from TMEM once; the
-//               running maximum is kept unless the tile exceeds it by more than 2^8 (then O_a and the
-//               row sum are rescaled first), P = 2^(s - m) goes back to TMEM as bf16 over S
-//   warps 4-7   the same for half b
-//   warp 8      TMA producer: K and V tiles of 128 keys through a shared-memory ring (Q and the first K, V
+// Blackwell.  The key range is walked 64 keys at a time, and a block is ONE softmax chain:
+//   logits ready -> softmax warpgroup -> P ready -> tensor core (O += P V, next logits) -> ...
+// A chain spends most of its time waiting for the other side (the round trip through the barriers and the
+// tensor core's queue is longer than either side's work), so what keeps an SM busy is the number of
+// independent chains on it: a block is kept small (192 threads, 128 TMEM columns, 50 KB of shared memory)
+// and FOUR blocks share an SM.  Each block's set-up, first copies and epilogue, during which it computes
+// nothing, are then overlapped by three running chains instead of being a quarter of its life.
+//   warps 0-3   softmax: one query row per thread, 64 logits per tile read from TMEM once; the running
+//               maximum is kept unless the tile exceeds it by more than 2^8 (then O and the row sum are
+//               rescaled first), P = 2^(s - m) goes back to TMEM as bf16 over S; at the end O / l -> out
+//   warp 4      TMA producer: K and V tiles of 64 keys through a shared-memory ring (Q and the first K, V
 //               tiles are requested by thread 0 during the set-up).  The tensor maps are 4-D (64, rows,
 //               heads, batches) with the tensor's own strides, so contiguous [B,H,L,64] tensors and the
 //               packed [B,L,3,H,64] projection output go through the same code; the output address is
 //               formed from three strides
-//   warp 9      issues tcgen05.mma: S_x = Q K_x^T (both operands in shared memory), O_x += P_x V_x (P_x from
-//               TMEM, V_x an MN-major shared-memory operand), one burst per half and tile:
-//               O_x += P_x V_x of tile j, then S_x of tile j + 1 into the columns P_x has just left
-// TMEM columns: S/P of half a [0,64), of half b [64,128), O_a [128,192), O_b [192,256).
-// Registers: the block starts with 80 per thread (two blocks per SM); the softmax warpgroups raise
-// theirs to 96 and the third warpgroup drops to 48 (setmaxnreg), the same total.
+//   warp 5      issues tcgen05.mma: S = Q K^T (both operands in shared memory), O += P V (P from TMEM, V an
+//               MN-major shared-memory operand), one burst per tile: O += P V of tile j, then S of tile
+//               j + 1 into the columns P has just left
+// TMEM columns: S/P [0,64), O [64,128).
+// Registers: the block starts with 80 per thread (four blocks per SM); the softmax warps raise theirs to
+// 96 and the other two warps drop to 48 (setmaxnreg), the same total.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -39,28 +39,27 @@ namespace {
 using namespace ptx;
 
 constexpr int BM = 128;              // query rows per block
-constexpr int BN = 128;              // keys per tile
-constexpr int HN = 64;               // keys per half tile
+constexpr int BN = 64;               // keys per tile
 constexpr int D = kHeadDim;
 constexpr int NSTAGE = 2;
-constexpr int TILE_BYTES = BN * D * 2;          // 16 KB
-constexpr int NUM_THREADS = 384;
-constexpr int NUM_SOFTMAX_THREADS = 256;
-constexpr int PRODUCER_WARP = 8, MMA_WARP = 9;
+constexpr int Q_BYTES = BM * D * 2;             // 16 KB
+constexpr int TILE_BYTES = BN * D * 2;          // 8 KB
+constexpr int NUM_THREADS = 192;
+constexpr int NUM_SOFTMAX_THREADS = 128;
+constexpr int PRODUCER_WARP = 4, MMA_WARP = 5;
 constexpr int REGS_START = 80, REGS_SOFTMAX = 96, REGS_MISC = 48;
-static_assert(2 * REGS_SOFTMAX + REGS_MISC == 3 * REGS_START, "register budget of the block");
-constexpr uint32_t TMEM_COLS = 256;
-constexpr uint32_t COL_S = 0, COL_O = 128;
+static_assert(4 * REGS_SOFTMAX + 2 * REGS_MISC == 6 * REGS_START, "register budget of the block");
+constexpr uint32_t TMEM_COLS = 128;
+constexpr uint32_t COL_S = 0, COL_O = 64;
 constexpr float kRescaleThreshold = 8.0f;       // in log2 units
 
 struct __align__(1024) SharedStorage {
-    uint8_t q[TILE_BYTES];
+    uint8_t q[Q_BYTES];
     uint8_t k[NSTAGE][TILE_BYTES];
     uint8_t v[NSTAGE][TILE_BYTES];
-    float2 stats[2][BM];                     // (running maximum, row sum) of each half, for the merge
     uint64_t q_full;
     uint64_t k_full[NSTAGE], k_empty[NSTAGE], v_full[NSTAGE], v_empty[NSTAGE];
-    uint64_t s_full[2], p_full[2], o_done, stats_ready;
+    uint64_t s_full, p_full, o_done;
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -68,7 +67,7 @@ struct __align__(1024) SharedStorage {
 struct KvTile {
     int seg;        // 0 or 1
     int coord;      // first row of the tile inside its tensor
-    int n_valid;    // valid keys in the tile (1..128)
+    int n_valid;    // valid keys in the tile (1..64)
 };
 
 __device__ __forceinline__ KvTile kv_tile(const FwdWork& w, int tiles0, int j) {
@@ -85,11 +84,8 @@ __device__ __forceinline__ KvTile kv_tile(const FwdWork& w, int tiles0, int j) {
     return t;
 }
 
-// columns issued for half h of a tile with n_valid keys (multiple of 16, 0 if the half is empty)
-__device__ __forceinline__ int half_cols(int n_valid, int h) {
-    const int n_eff = (n_valid + 15) & ~15;
-    return h == 0 ? min(n_eff, HN) : max(n_eff - HN, 0);
-}
+// columns issued for a tile with n_valid keys (a multiple of 16)
+__device__ __forceinline__ int tile_cols(int n_valid) { return (n_valid + 15) & ~15; }
 
 __device__ __forceinline__ void report_timeout(int* status, int where) {
     if (status != nullptr) {
@@ -105,7 +101,7 @@ template <int N> __device__ __forceinline__ void reg_dec() {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
 
-__global__ void __launch_bounds__(NUM_THREADS, 2)
+__global__ void __launch_bounds__(NUM_THREADS, 4)
 hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k0,
                    const __grid_constant__ CUtensorMap map_v0, const __grid_constant__ CUtensorMap map_k1,
                    const __grid_constant__ CUtensorMap map_v1, const FwdArgs args) {
@@ -146,17 +142,14 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             mbar_init(&sm.v_full[s], 1);
             mbar_init(&sm.v_empty[s], 1);
         }
-        for (int h = 0; h < 2; ++h) {
-            mbar_init(&sm.s_full[h], 1);
-            mbar_init(&sm.p_full[h], NUM_SOFTMAX_THREADS / 2);
-        }
+        mbar_init(&sm.s_full, 1);
+        mbar_init(&sm.p_full, NUM_SOFTMAX_THREADS);
         mbar_init(&sm.o_done, 1);
-        mbar_init(&sm.stats_ready, NUM_SOFTMAX_THREADS);
         fence_mbar_init();
         // The block's first copies (Q, first K and V tiles) start here, before the TMEM allocation and the
         // block-wide barrier, so that their latency overlaps the rest of the set-up.
         const KvTile t0 = kv_tile(w, tiles0, 0);
-        mbar_arrive_expect_tx(&sm.q_full, TILE_BYTES);
+        mbar_arrive_expect_tx(&sm.q_full, Q_BYTES);
         tma_load_4d(sm.q, &map_q, &sm.q_full, 0, w.row_begin, head, batch);
         mbar_arrive_expect_tx(&sm.k_full[0], TILE_BYTES);
         tma_load_4d(sm.k[0], t0.seg ? &map_k1 : &map_k0, &sm.k_full[0], 0, t0.coord, head, batch);
@@ -174,7 +167,6 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     volatile int* abort_flag = &sm.abort_flag;
 
     if (warp >= PRODUCER_WARP) {
-        reg_dec<REGS_MISC>();
         if (warp == PRODUCER_WARP) {
             // ================================================================== TMA producer
             // The whole warp runs the control flow; one elected lane issues the copies (a warp that has split
@@ -211,41 +203,38 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 const uint64_t t0 = globaltimer_ns();
                 while (globaltimer_ns() - t0 < 2000000ull) { }
             }
-        } else if (warp == MMA_WARP) {
+        } else {
             // ================================================================== MMA issuer
             // The whole warp runs the control flow; one elected lane issues.  Descriptors are built once and
             // advanced by adding (byte offset >> 4), so issuing an MMA costs a few instructions.
             const bool leader = elect_one();
             const uint64_t q_kd = smem_desc_sw128(smem_u32(sm.q), 16);
-            const uint64_t k_kd0 = smem_desc_sw128(smem_u32(sm.k[0]), 16);      // ring slots are 16 KB apart
+            const uint64_t k_kd0 = smem_desc_sw128(smem_u32(sm.k[0]), 16);      // ring slots are 8 KB apart
             const uint64_t v_mn0 = smem_desc_sw128(smem_u32(sm.v[0]), 1024);
             constexpr uint32_t idesc_pv = idesc_bf16_f32(BM, D, false, true);
-            uint32_t par_p[2] = {0, 0};                             // parity of the next p_full[h] phase
-            bool o_started[2] = {false, false};                     // O_x has received a product
+            constexpr uint32_t SLOT_UNITS = TILE_BYTES >> 4;
             auto wait = [&](uint64_t* bar, uint32_t parity, int code) -> bool {
                 if (__all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag))) return true;
                 if (lane == 0) report_timeout(args.status, code);
                 return false;
             };
-            // S_h = Q K_h^T for n keys of half h of the tile in ring slot `slot`
-            auto issue_s = [&](int h, int n, int slot) {
+            // S = Q K^T for n keys of the tile in ring slot `slot`
+            auto issue_s = [&](int n, int slot) {
                 const uint32_t idesc = idesc_bf16_f32(BM, n, false, false);
-                const uint64_t kd = k_kd0 + slot * 1024 + h * 512;              // + 64 rows
+                const uint64_t kd = k_kd0 + slot * SLOT_UNITS;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks)
-                    mma_ss(tmem + COL_S + h * HN, q_kd + ks * 2, kd + ks * 2, idesc, ks > 0);
-                tc_commit(&sm.s_full[h]);
+                    mma_ss(tmem + COL_S, q_kd + ks * 2, kd + ks * 2, idesc, ks > 0);
+                tc_commit(&sm.s_full);
             };
-            // O_h += P_h V_h for n keys of half h
-            auto issue_pv = [&](int h, int n, int slot) {
+            // O += P V for n keys
+            auto issue_pv = [&](int n, int slot, bool first) {
                 const int nk = n / 16;
-                const uint64_t vd = v_mn0 + slot * 1024 + h * 512;
+                const uint64_t vd = v_mn0 + slot * SLOT_UNITS;
 #pragma unroll
-                for (int ks = 0; ks < HN / 16; ++ks)
+                for (int ks = 0; ks < BN / 16; ++ks)
                     if (ks < nk)
-                        mma_ts(tmem + COL_O + h * HN, tmem + COL_S + h * HN + ks * 8, vd + ks * 128, idesc_pv,
-                               o_started[h] || (ks > 0));
-                o_started[h] = true;
+                        mma_ts(tmem + COL_O, tmem + COL_S + ks * 8, vd + ks * 128, idesc_pv, !first || (ks > 0));
             };
 
             bool ok = true;
@@ -256,10 +245,8 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
             if (ok) {
                 tc_fence_after();
-                const int nv = kv_tile(w, tiles0, 0).n_valid;
                 if (leader) {
-                    issue_s(0, half_cols(nv, 0), 0);
-                    if (half_cols(nv, 1) > 0) issue_s(1, half_cols(nv, 1), 0);
+                    issue_s(tile_cols(kv_tile(w, tiles0, 0).n_valid), 0);
                     if (NSTAGE < n_tiles) tc_commit(&sm.k_empty[0]);
                 }
                 __syncwarp();
@@ -267,55 +254,40 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             for (int j = 0; j < n_tiles && ok; ++j) {
                 const int slot = j % NSTAGE, slot_next = (j + 1) % NSTAGE;
                 const bool more = j + 1 < n_tiles;
-                const int nv = kv_tile(w, tiles0, j).n_valid;
-                const int nv_next = more ? kv_tile(w, tiles0, j + 1).n_valid : 0;
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int n = half_cols(nv, h), n_next = half_cols(nv_next, h);
-                    // one burst: O_h += P_h V_h of tile j, then S_h of tile j + 1 over the columns P_h leaves.
-                    // The copies are looked at first (normally long complete): a look at a barrier is a
-                    // shared-memory round trip behind the softmax warps' traffic, and after the softmax
-                    // warpgroup's arrival every such trip delays the products it is waiting for.
-                    if (h == 0) {
-                        // both looks are sent before either answer is used
-                        const bool rv = mbar_try_wait(&sm.v_full[slot], (j / NSTAGE) & 1);
-                        const bool rk = !more || mbar_try_wait(&sm.k_full[slot_next], ((j + 1) / NSTAGE) & 1);
-                        if (!__all_sync(0xffffffffu, rv && rk))
-                            ok = (rv || wait(&sm.v_full[slot], (j / NSTAGE) & 1, 0x500 + j)) &&
-                                 (rk || wait(&sm.k_full[slot_next], ((j + 1) / NSTAGE) & 1, 0x400 + j));
-                    }
-                    if (ok && n > 0) {
-                        ok = wait(&sm.p_full[h], par_p[h], 0x600 + j);
-                        par_p[h] ^= 1;
-                    }
-                    if (!ok) break;
-                    tc_fence_after();
-                    if (leader) {
-                        if (n > 0) issue_pv(h, n, slot);
-                        if (n_next > 0) issue_s(h, n_next, slot_next);
-                        if (h == 1) {
-                            // V of tile j and K of tile j + 1 have been handed to their last readers; a slot is
-                            // signalled free only if a later tile will use it (the block may exit as soon as the
-                            // softmax warps have seen o_done: an arrival that lands after that would hit the
-                            // barriers of the next block on this SM)
-                            if (j + NSTAGE < n_tiles) tc_commit(&sm.v_empty[slot]);
-                            if (j + 1 + NSTAGE < n_tiles) tc_commit(&sm.k_empty[slot_next]);
-                            if (!more) tc_commit(&sm.o_done);
-                        }
-                    } else if (n > 0) {
-                        o_started[h] = true;
-                    }
-                    __syncwarp();
+                const int n = tile_cols(kv_tile(w, tiles0, j).n_valid);
+                const int n_next = more ? tile_cols(kv_tile(w, tiles0, j + 1).n_valid) : 0;
+                // one burst: O += P V of tile j, then S of tile j + 1 over the columns P leaves.  The copies are
+                // looked at first (normally long complete), both looks sent before either answer is used: a look
+                // at a barrier is a shared-memory round trip, and after the softmax warps' arrival every such trip
+                // delays the products they are waiting for.
+                {
+                    const bool rv = mbar_try_wait(&sm.v_full[slot], (j / NSTAGE) & 1);
+                    const bool rk = !more || mbar_try_wait(&sm.k_full[slot_next], ((j + 1) / NSTAGE) & 1);
+                    if (!__all_sync(0xffffffffu, rv && rk))
+                        ok = (rv || wait(&sm.v_full[slot], (j / NSTAGE) & 1, 0x500 + j)) &&
+                             (rk || wait(&sm.k_full[slot_next], ((j + 1) / NSTAGE) & 1, 0x400 + j));
                 }
+                if (ok) ok = wait(&sm.p_full, j & 1, 0x600 + j);
+                if (!ok) break;
+                tc_fence_after();
+                if (leader) {
+                    issue_pv(n, slot, j == 0);
+                    if (n_next > 0) issue_s(n_next, slot_next);
+                    // V of tile j and K of tile j + 1 have been handed to their last readers; a slot is signalled
+                    // free only if a later tile will use it (the block may exit as soon as the softmax warps have
+                    // seen o_done: an arrival that lands after that would hit the barriers of the next block on
+                    // this SM)
+                    if (j + NSTAGE < n_tiles) tc_commit(&sm.v_empty[slot]);
+                    if (j + 1 + NSTAGE < n_tiles) tc_commit(&sm.k_empty[slot_next]);
+                    if (!more) tc_commit(&sm.o_done);
+                }
+                __syncwarp();
             }
         }
     } else {
-        // ================================================================== softmax warpgroups + epilogue
-        reg_inc<REGS_SOFTMAX>();
-        const int quarter = warp & 3;
-        const int h = warp >> 2;                               // the half of every tile this warpgroup owns
-        const int r = quarter * 32 + lane;                     // row inside the tile
-        const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+        // ================================================================== softmax warps + epilogue
+        const int r = warp * 32 + lane;                        // row inside the tile
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
         const int row = w.row_begin + r;
         const bool row_ok = r < w.row_count;
         int lo = w.s0_begin, hi = w.s0_end;                    // per-row key bounds (training, packed tiles)
@@ -325,40 +297,36 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             hi = args.st.start[s + 1];
         }
         const float sl2 = args.scale_log2;
-        const int col0 = h * HN;                               // first key of this half inside a tile
-        const uint32_t s_addr = lane_base + COL_S + col0;
-        const uint32_t o_addr = lane_base + COL_O + col0;
+        const uint32_t s_addr = lane_base + COL_S;
+        const uint32_t o_addr = lane_base + COL_O;
         float m_used = -INFINITY, l = 0.f;
         bool ok = true;
-        bool have_o = false;                                   // O_h has received a product
-        uint32_t par_s = 0;                                    // parity of the next s_full[h] phase
         uint32_t b0[32], b1[32];
 
         for (int j = 0; j < n_tiles && ok; ++j) {
             const KvTile t = kv_tile(w, tiles0, j);
-            const int n = half_cols(t.n_valid, h);
-            if (n == 0) continue;
+            const int n = tile_cols(t.n_valid);
             // key c of the tile is visible to this row iff c in [c_lo, c_hi)
             const int c_lo = w.uniform ? 0 : max(lo - t.coord, 0);
             const int c_hi = w.uniform ? t.n_valid : min(hi - t.coord, t.n_valid);
             const bool two = n > 32;                           // second 32-column chunk present
-            const bool need_mask = (!w.uniform) || (t.n_valid < col0 + (two ? 64 : 32));
+            const bool need_mask = (!w.uniform) || (t.n_valid < (two ? 64 : 32));
 
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[h], par_s, abort_flag));
+            ok = __all_sync(0xffffffffu, mbar_wait(&sm.s_full, j & 1, abort_flag));
             if (!ok) { if (lane == 0) report_timeout(args.status, 0x800 + j); break; }
-            par_s ^= 1;
             tc_fence_after();
 
             tmem_ld32(s_addr, b0);
             if (two) tmem_ld32(s_addr + 32, b1);
             tmem_ld_wait();
 
-            // masked logits become -inf once, so the maximum and the exponentials treat them alike
+            // masked logits become -inf once, so the maximum and the exponentials treat them alike (columns the
+            // tensor core did not write hold stale values and lie outside [c_lo, c_hi) too)
             if (need_mask) {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
-                    if (!(col0 + i >= c_lo && col0 + i < c_hi)) b0[i] = 0xff800000u;
-                    if (!(col0 + 32 + i >= c_lo && col0 + 32 + i < c_hi)) b1[i] = 0xff800000u;
+                    if (!(i >= c_lo && i < c_hi)) b0[i] = 0xff800000u;
+                    if (!(32 + i >= c_lo && 32 + i < c_hi)) b1[i] = 0xff800000u;
                 }
             }
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};     // four chains of maxima, not one of 64
@@ -370,16 +338,16 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             }
             const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sl2;     // softmax_scale > 0
 
-            // Keep the running maximum unless this tile exceeds it by more than the threshold.  O_h is
-            // quiet here: the product that precedes S_h of this tile in the tensor core's queue is the
-            // last one that wrote it, and the next one waits for this warpgroup.
+            // Keep the running maximum unless this tile exceeds it by more than the threshold.  O is quiet
+            // here: the product that precedes S of this tile in the tensor core's queue is the last one that
+            // wrote it, and the next one waits for these warps.
             const bool grow = mx > m_used + kRescaleThreshold;  // false for -inf > -inf
             if (__any_sync(0xffffffffu, grow)) {
                 const float m_new = fmaxf(m_used, mx);
                 const float f = (m_used == -INFINITY) ? 0.f : ex2(m_used - m_new);
                 m_used = m_new;
                 l *= f;
-                if (have_o) {
+                if (j > 0) {
 #pragma unroll 1
                     for (int piece = 0; piece < 4; ++piece) {
                         uint32_t o[16];
@@ -417,58 +385,44 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             l += l_add;
             tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(&sm.p_full[h]);
-            have_o = true;
+            mbar_arrive(&sm.p_full);
         }
 
-        // ---- merge of the two halves and epilogue: this warpgroup writes output columns [32 h, 32 h + 32)
-        // (the row statistics are final once the last P is out: they are exchanged while the last products run)
-        if (ok) {
-            sm.stats[h][r] = make_float2(m_used, l);
-            mbar_arrive(&sm.stats_ready);
-            ok = __all_sync(0xffffffffu, mbar_wait(&sm.stats_ready, 0, abort_flag));
-            if (!ok && lane == 0) report_timeout(args.status, 0xB00);
-        }
+        // ---- epilogue: out = O / l, lse = ln(l) + m (natural log of the scaled logits' sum)
         if (ok) {
             ok = __all_sync(0xffffffffu, mbar_wait(&sm.o_done, 0, abort_flag));
             if (!ok && lane == 0) report_timeout(args.status, 0xA00);
         }
         if (ok) {
             tc_fence_after();
-            const float2 sa = sm.stats[0][r], sb = sm.stats[1][r];
-            // half a always has keys; half b has none when every tile of the block is at most 64 keys wide
-            // (its accumulator is then unwritten and must not be read into the result)
-            const bool b_used = sb.y > 0.f;
-            const float m = b_used ? fmaxf(sa.x, sb.x) : sa.x;
-            const float wa = ex2(sa.x - m);
-            const float wb = b_used ? ex2(sb.x - m) : 0.f;
-            const float lsum = sa.y * wa + sb.y * wb;
-            const float inv = 1.f / lsum;
-            const float fa = wa * inv, fb = wb * inv;
-            tmem_ld32(lane_base + COL_O + h * 32, b0);                 // O_a, this warpgroup's 32 columns
-            tmem_ld32(lane_base + COL_O + HN + h * 32, b1);            // O_b
+            const float inv = 1.f / l;
+            tmem_ld32(o_addr, b0);
+            tmem_ld32(o_addr + 32, b1);
             tmem_ld_wait();
             if (row_ok) {
                 __nv_bfloat16* orow = args.out + batch * args.out_batch_stride + head * args.out_head_stride +
-                                      row * args.out_row_stride + h * 32;
+                                      row * args.out_row_stride;
                 uint4* dst = reinterpret_cast<uint4*>(orow);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    float o[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        const float a = __uint_as_float(b0[8 * i + e]) * fa;
-                        o[e] = b_used ? fmaf(__uint_as_float(b1[8 * i + e]), fb, a) : a;
-                    }
                     uint4 v4;
-                    v4.x = pack_bf16(o[0], o[1]);
-                    v4.y = pack_bf16(o[2], o[3]);
-                    v4.z = pack_bf16(o[4], o[5]);
-                    v4.w = pack_bf16(o[6], o[7]);
+                    v4.x = pack_bf16(__uint_as_float(b0[8 * i + 0]) * inv, __uint_as_float(b0[8 * i + 1]) * inv);
+                    v4.y = pack_bf16(__uint_as_float(b0[8 * i + 2]) * inv, __uint_as_float(b0[8 * i + 3]) * inv);
+                    v4.z = pack_bf16(__uint_as_float(b0[8 * i + 4]) * inv, __uint_as_float(b0[8 * i + 5]) * inv);
+                    v4.w = pack_bf16(__uint_as_float(b0[8 * i + 6]) * inv, __uint_as_float(b0[8 * i + 7]) * inv);
                     dst[i] = v4;
                 }
-                if (h == 0 && args.lse != nullptr)
-                    args.lse[(size_t)bh * args.n_q_rows + row] = (m + log2f(lsum)) * 0.6931471805599453f;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    uint4 v4;
+                    v4.x = pack_bf16(__uint_as_float(b1[8 * i + 0]) * inv, __uint_as_float(b1[8 * i + 1]) * inv);
+                    v4.y = pack_bf16(__uint_as_float(b1[8 * i + 2]) * inv, __uint_as_float(b1[8 * i + 3]) * inv);
+                    v4.z = pack_bf16(__uint_as_float(b1[8 * i + 4]) * inv, __uint_as_float(b1[8 * i + 5]) * inv);
+                    v4.w = pack_bf16(__uint_as_float(b1[8 * i + 6]) * inv, __uint_as_float(b1[8 * i + 7]) * inv);
+                    dst[4 + i] = v4;
+                }
+                if (args.lse != nullptr)
+                    args.lse[(size_t)bh * args.n_q_rows + row] = (m_used + log2f(l)) * 0.6931471805599453f;
             }
         }
     }

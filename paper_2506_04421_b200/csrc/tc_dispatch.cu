@@ -51,15 +51,16 @@ static bool make_rows_map(CUtensorMap* map, const void* base, int heads, int row
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 4-D map (64 elements, rows, heads, batches) with the strides of the tensor in elements; boxes of 128 rows
-// of one head.  Serves the contiguous [B, H, rows, 64] layout and a packed [B, rows, 3, H, 64] one alike.
+// 4-D map (64 elements, rows, heads, batches) with the strides of the tensor in elements; boxes of `box_rows`
+// rows of one head.  Serves the contiguous [B, H, rows, 64] layout and a packed [B, rows, 3, H, 64] one alike.
+constexpr int kFwdKeyRows = 64;      // key rows per tile of the forward kernel (its query tiles are kTileRows high)
 static bool make_rows_map4(CUtensorMap* map, const void* base, int batches, int heads, int rows, long long row_stride,
-                           long long head_stride, long long batch_stride) {
+                           long long head_stride, long long batch_stride, int box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (fn == nullptr) return false;
     const cuuint64_t dims[4] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows, (cuuint64_t)heads, (cuuint64_t)batches};
     const cuuint64_t strides[3] = {(cuuint64_t)row_stride * 2, (cuuint64_t)head_stride * 2, (cuuint64_t)batch_stride * 2};
-    const cuuint32_t box[4] = {(cuuint32_t)kHeadDim, (cuuint32_t)kTileRows, 1, 1};
+    const cuuint32_t box[4] = {(cuuint32_t)kHeadDim, (cuuint32_t)box_rows, 1, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -176,8 +177,9 @@ static int tc_fwd_strided(const bf16* q, const bf16* k, const bf16* v, bf16* out
     if (plan == nullptr) return HMAR_ERR_CUDA;
     const int L = st.start[st.n_scales];
     CUtensorMap mq, mk, mv;
-    if (!make_rows_map4(&mq, q, B, H, L, in_row, in_head, in_batch) || !make_rows_map4(&mk, k, B, H, L, in_row, in_head, in_batch) ||
-        !make_rows_map4(&mv, v, B, H, L, in_row, in_head, in_batch))
+    if (!make_rows_map4(&mq, q, B, H, L, in_row, in_head, in_batch, kTileRows) ||
+        !make_rows_map4(&mk, k, B, H, L, in_row, in_head, in_batch, kFwdKeyRows) ||
+        !make_rows_map4(&mv, v, B, H, L, in_row, in_head, in_batch, kFwdKeyRows))
         return HMAR_ERR_CUDA;
     FwdArgs a{};
     a.work = plan->fwd_work;
@@ -220,13 +222,15 @@ int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const b
         return step_small(q, k_prev, v_prev, k_cur, v_cur, out, lse, BH, n_prev, n_cur, st.q, st.kv_prev, st.kv_cur, st.out,
                           scale, stream);
     CUtensorMap mq, mk0, mv0, mk1, mv1;
-    auto rows_map = [&](CUtensorMap* m, const bf16* base, int rows, long long head_stride) {
-        return make_rows_map4(m, base, 1, BH, rows, kHeadDim, head_stride, (long long)BH * head_stride);
+    auto rows_map = [&](CUtensorMap* m, const bf16* base, int rows, long long head_stride, int box_rows) {
+        return make_rows_map4(m, base, 1, BH, rows, kHeadDim, head_stride, (long long)BH * head_stride, box_rows);
     };
-    if (!rows_map(&mq, q, n_cur, st.q) || !rows_map(&mk1, k_cur, n_cur, st.kv_cur) || !rows_map(&mv1, v_cur, n_cur, st.kv_cur))
+    if (!rows_map(&mq, q, n_cur, st.q, kTileRows) || !rows_map(&mk1, k_cur, n_cur, st.kv_cur, kFwdKeyRows) ||
+        !rows_map(&mv1, v_cur, n_cur, st.kv_cur, kFwdKeyRows))
         return HMAR_ERR_CUDA;
     if (n_prev > 0) {
-        if (!rows_map(&mk0, k_prev, n_prev, st.kv_prev) || !rows_map(&mv0, v_prev, n_prev, st.kv_prev)) return HMAR_ERR_CUDA;
+        if (!rows_map(&mk0, k_prev, n_prev, st.kv_prev, kFwdKeyRows) || !rows_map(&mv0, v_prev, n_prev, st.kv_prev, kFwdKeyRows))
+            return HMAR_ERR_CUDA;
     } else {
         mk0 = mk1;
         mv0 = mv1;
