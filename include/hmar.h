@@ -49,15 +49,18 @@ typedef enum {
 
 #define HMAR_MAX_SCALES 64
 
-/* Which scales a token of scale k attends to.  All three are block masks over the same flattened
+/* Which scales a token of scale k attends to.  All four are block masks over the same flattened
  * sequence in which the allowed keys of a query are one contiguous range, so one scheduler and one set
  * of kernels serves them.
  *   HMAR_WINDOW_MARKOV : scales k-1 and k - HMAR's Markovian mask (Sec. 4.1, Fig. attn-mask); what the
  *                        entry points without `_window` compute.
  *   HMAR_WINDOW_CAUSAL : scales 1..k - VAR's block-causal mask (Sec. 3, Fig. attn-mask), the workload the
  *                        paper's attention benchmark compares against (App. B.4).
- *   HMAR_WINDOW_SELF   : scale k only - the literal "block-diagonal" reading of Sec. 1 / App. B.3. */
-typedef enum { HMAR_WINDOW_MARKOV = 0, HMAR_WINDOW_CAUSAL = 1, HMAR_WINDOW_SELF = 2 } hmar_window;
+ *   HMAR_WINDOW_SELF   : scale k only - the literal "block-diagonal" reading of Sec. 1 / App. B.3.
+ *   HMAR_WINDOW_PREV   : scale k-1 only - App. B.3's literal "only the immediately preceding scale"; the first
+ *                        scale, which has no predecessor, attends to itself.  No query looks at the keys of the
+ *                        last scale, so the backward returns zeros for their dK and dV. */
+typedef enum { HMAR_WINDOW_MARKOV = 0, HMAR_WINDOW_CAUSAL = 1, HMAR_WINDOW_SELF = 2, HMAR_WINDOW_PREV = 3 } hmar_window;
 
 /* Training forward (Sec. 4.1; App. B.4 benchmarks this pass).
  *   q, k, v : [B,H,L,D] in;  out : [B,H,L,D] out;  lse : [B,H,L] fp32 out.

@@ -70,16 +70,27 @@ def block_diagonal_mask(side_lens):
     return s[None, :] == s[:, None]
 
 
+def previous_scale_mask(side_lens):
+    """Scale k attends to scale k-1 only (App. B.3 read literally: "only the immediately preceding scale");
+    the first scale has no predecessor and attends to itself, so that no row is empty."""
+    s = scale_of_token(side_lens)
+    si = s[:, None]
+    sj = s[None, :]
+    return (sj == si - 1) | ((si == 0) & (sj == 0))
+
+
 def window_mask(side_lens, window="markov"):
     """The mask of the family named by `window`: "markov" (HMAR, scales k-1 and k), "causal" (VAR's
-    block-causal mask, Sec. 3) or "self" (block-diagonal)."""
+    block-causal mask, Sec. 3), "self" (block-diagonal) or "prev" (the preceding scale only)."""
     if window == "markov":
         return hmar_mask(side_lens)
     if window == "causal":
         return block_causal_mask(side_lens)
     if window == "self":
         return block_diagonal_mask(side_lens)
-    raise ValueError("window must be 'markov', 'causal' or 'self'")
+    if window == "prev":
+        return previous_scale_mask(side_lens)
+    raise ValueError("window must be 'markov', 'causal', 'self' or 'prev'")
 
 
 def count_pairs(side_lens, window="markov"):

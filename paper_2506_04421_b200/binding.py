@@ -24,6 +24,7 @@ HMAR_ERR_DEVICE_TIMEOUT = -5
 HMAR_WINDOW_MARKOV = 0      # scales k-1 and k (HMAR)
 HMAR_WINDOW_CAUSAL = 1      # scales 1..k (VAR's block-causal mask)
 HMAR_WINDOW_SELF = 2        # scale k only (block-diagonal)
+HMAR_WINDOW_PREV = 3        # scale k-1 only; the first scale attends to itself
 
 EXPORTED_SYMBOLS = (
     "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_fwd_window", "hmar_attn_fwd_window_f32", "hmar_attn_fwd_packed",

@@ -67,7 +67,7 @@ static int check_shape(int B, int H, int D) {
 
 static int check_sides(int n_scales, const int* side_lens, int window, ScaleTable* st) {
     if (n_scales <= 0 || n_scales > HMAR_MAX_SCALES || side_lens == nullptr) return HMAR_ERR_BAD_ARG;
-    if (window != HMAR_WINDOW_MARKOV && window != HMAR_WINDOW_CAUSAL && window != HMAR_WINDOW_SELF) return HMAR_ERR_BAD_ARG;
+    if (window < HMAR_WINDOW_MARKOV || window > HMAR_WINDOW_PREV) return HMAR_ERR_BAD_ARG;
     long long total = 0;
     for (int s = 0; s < n_scales; ++s) {
         if (side_lens[s] <= 0 || side_lens[s] > 4096) return HMAR_ERR_BAD_ARG;

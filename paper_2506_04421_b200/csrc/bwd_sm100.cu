@@ -709,7 +709,7 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     if (rr >= w.row_count) { qlo[i] = 0; qhi[i] = 0; }
                     else if (!w.uniform) {
                         const int sc = scale_of_row(args.st, w.row_begin + rr);
-                        qlo[i] = args.st.start[sc];
+                        qlo[i] = args.st.start[first_query_scale(args.st.window, sc)];
                         qhi[i] = args.st.start[last_query_scale(args.st.window, sc, args.st.n_scales) + 1];
                     }
                 }

@@ -294,7 +294,7 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         if (!w.uniform && row_ok) {
             const int s = scale_of_row(args.st, row);
             lo = args.st.start[first_key_scale(args.st.window, s)];
-            hi = args.st.start[s + 1];
+            hi = args.st.start[last_key_scale(args.st.window, s) + 1];
         }
         const float sl2 = args.scale_log2;
         const uint32_t s_addr = lane_base + COL_S;

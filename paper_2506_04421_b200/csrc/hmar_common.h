@@ -21,10 +21,18 @@ struct ScaleTable {
 #else
 #define HMAR_HD inline
 #endif
-// The keys a query of scale s sees are the scales first_key_scale(s) .. s, a contiguous range of the
-// flattened sequence; the queries that see a key of scale s are the scales s .. last_query_scale(s).
+// The keys a query of scale s sees are the scales first_key_scale(s) .. last_key_scale(s), a contiguous range of
+// the flattened sequence; the queries that see a key of scale s are the scales first_query_scale(s) ..
+// last_query_scale(s), also contiguous - and empty (first > last) for the keys of the last scale under
+// HMAR_WINDOW_PREV, which no query looks at.
 HMAR_HD int first_key_scale(int window, int s) {
     return window == HMAR_WINDOW_CAUSAL ? 0 : (window == HMAR_WINDOW_SELF ? s : (s > 0 ? s - 1 : 0));
+}
+HMAR_HD int last_key_scale(int window, int s) {
+    return (window == HMAR_WINDOW_PREV && s > 0) ? s - 1 : s;
+}
+HMAR_HD int first_query_scale(int window, int s) {
+    return (window == HMAR_WINDOW_PREV && s > 0) ? s + 1 : s;       // may be n_scales: no query sees the key
 }
 HMAR_HD int last_query_scale(int window, int s, int n_scales) {
     return window == HMAR_WINDOW_CAUSAL ? n_scales - 1 : (window == HMAR_WINDOW_SELF ? s : (s + 1 < n_scales ? s + 1 : s));
@@ -42,8 +50,8 @@ struct Tile {
     int32_t cost;      // number of kTileRows-wide partner tiles (for ordering)
 };
 
-// Forward bounds of query row `i` of scale s: keys [start[first_key_scale(s)], start[s+1]).
-// Backward bounds of key row `j` of scale s: queries [start[s], start[last_query_scale(s)+1]).
+// Forward bounds of query row `i` of scale s: keys [start[first_key_scale(s)], start[last_key_scale(s)+1]).
+// Backward bounds of key row `j` of scale s: queries [start[first_query_scale(s)], start[last_query_scale(s)+1]).
 void build_scale_table(int n_scales, const int* side_lens, int window, ScaleTable* out);
 std::vector<Tile> build_tiles(const ScaleTable& st, int direction);
 

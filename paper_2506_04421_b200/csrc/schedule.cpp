@@ -24,10 +24,11 @@ static void partner_range(const ScaleTable& st, int direction, int s_first, int 
     const int K = st.n_scales;
     if (direction == 0) {           // queries of scales s_first..s_last -> keys
         *begin = st.start[first_key_scale(st.window, s_first)];
-        *end = st.start[s_last + 1];
-    } else {                        // keys of scales s_first..s_last -> queries
-        *begin = st.start[s_first];
+        *end = st.start[last_key_scale(st.window, s_last) + 1];
+    } else {                        // keys of scales s_first..s_last -> queries (possibly none)
+        *begin = st.start[first_query_scale(st.window, s_first)];
         *end = st.start[last_query_scale(st.window, s_last, K) + 1];
+        if (*end < *begin) *end = *begin;
     }
 }
 
@@ -39,7 +40,13 @@ std::vector<Tile> build_tiles(const ScaleTable& st, int direction) {
         t.row_begin = row_begin;
         t.row_count = row_count;
         partner_range(st, direction, s_first, s_last, &t.partner_begin, &t.partner_end);
-        t.uniform = (s_first == s_last) ? 1 : 0;
+        // uniform: every scale of the tile has the whole partner range as its own
+        t.uniform = 1;
+        for (int s = s_first; s <= s_last; ++s) {
+            int b, e;
+            partner_range(st, direction, s, s, &b, &e);
+            if (b != t.partner_begin || e != t.partner_end) t.uniform = 0;
+        }
         t.cost = (t.partner_end - t.partner_begin + kTileRows - 1) / kTileRows;
         tiles.push_back(t);
     };

@@ -72,10 +72,10 @@ simt_fwd_kernel(const T* __restrict__ q, const T* __restrict__ k0, const T* __re
     } else {
         int s = scale_of_row(st, row);
         lo = st.start[first_key_scale(st.window, s)];
-        hi = st.start[s + 1];
+        hi = st.start[last_key_scale(st.window, s) + 1];
         int sf = scale_of_row(st, row0), sl = scale_of_row(st, last_row);
         blk_lo = st.start[first_key_scale(st.window, sf)];
-        blk_hi = st.start[sl + 1];
+        blk_hi = st.start[last_key_scale(st.window, sl) + 1];
     }
 
     float qr[DH], o[DH];
@@ -157,9 +157,9 @@ simt_dq_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
     const int row = row_ok ? row_raw : L - 1;
     const int last_row = min(row0 + ROWS, L) - 1;
     const int s_row = scale_of_row(st, row);
-    const int lo = st.start[first_key_scale(st.window, s_row)], hi = st.start[s_row + 1];
+    const int lo = st.start[first_key_scale(st.window, s_row)], hi = st.start[last_key_scale(st.window, s_row) + 1];
     const int sf = scale_of_row(st, row0), sl = scale_of_row(st, last_row);
-    const int blk_lo = st.start[first_key_scale(st.window, sf)], blk_hi = st.start[sl + 1];
+    const int blk_lo = st.start[first_key_scale(st.window, sf)], blk_hi = st.start[last_key_scale(st.window, sl) + 1];
     const size_t head = (size_t)bh * L;
 
     float qr[DH], gr[DH], acc[DH];
@@ -223,9 +223,10 @@ simt_dkdv_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __re
     const int last_row = min(row0 + ROWS, L) - 1;
     const int K = st.n_scales;
     const int s_row = scale_of_row(st, row);
-    const int lo = st.start[s_row], hi = st.start[last_query_scale(st.window, s_row, K) + 1];
-    const int blk_lo = st.start[scale_of_row(st, row0)];
-    const int blk_hi = st.start[last_query_scale(st.window, scale_of_row(st, last_row), K) + 1];
+    // (under HMAR_WINDOW_PREV the keys of the last scale have no queries: lo = hi = L, and dK = dV = 0 is stored)
+    const int lo = st.start[first_query_scale(st.window, s_row)], hi = max(lo, st.start[last_query_scale(st.window, s_row, K) + 1]);
+    const int blk_lo = st.start[first_query_scale(st.window, scale_of_row(st, row0))];
+    const int blk_hi = max(blk_lo, st.start[last_query_scale(st.window, scale_of_row(st, last_row), K) + 1]);
     const size_t head = (size_t)bh * L;
 
     float kr[DH], vr[DH], ak[DH], av[DH];

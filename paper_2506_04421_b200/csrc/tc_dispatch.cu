@@ -3,6 +3,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <map>
 #include <mutex>
 #include <vector>
@@ -89,6 +90,7 @@ struct Plan {
     int n_fwd = 0;
     int n_bwd = 0;
     int bwd_head_cost = 0;
+    int zero_begin = 0, zero_end = 0;   // key rows of a head that no query sees: their dK, dV are zeros
 };
 
 struct PlanKey {
@@ -123,6 +125,20 @@ static const Plan* get_plan(const ScaleTable& st) {
         work[i].pad = 0;
     }
     std::vector<Tile> btiles = build_tiles(st, 1);
+    // Key tiles that no query sees (the last scale under HMAR_WINDOW_PREV) are not work items: the backward
+    // kernel's pipeline wants at least one step per item.  Their rows are one stretch at the end of the head.
+    Plan plan;
+    {
+        std::vector<Tile> live;
+        plan.zero_begin = plan.zero_end = 0;
+        for (const Tile& t : btiles) {
+            if (t.partner_end > t.partner_begin) { live.push_back(t); continue; }
+            if (plan.zero_end == plan.zero_begin) { plan.zero_begin = t.row_begin; plan.zero_end = t.row_begin + t.row_count; }
+            plan.zero_begin = std::min(plan.zero_begin, (int)t.row_begin);
+            plan.zero_end = std::max(plan.zero_end, (int)(t.row_begin + t.row_count));
+        }
+        btiles.swap(live);
+    }
     std::vector<BwdWork> bwork(btiles.size());
     for (size_t i = 0; i < btiles.size(); ++i) {
         bwork[i] = BwdWork{};
@@ -133,7 +149,6 @@ static const Plan* get_plan(const ScaleTable& st) {
         bwork[i].uniform = btiles[i].uniform;
     }
     static_assert(sizeof(FwdWork) == sizeof(BwdWork), "work tiles share one allocation");
-    Plan plan;
     plan.bwd_head_cost = bwd_fill_costs(bwork.data(), (int)bwork.size());
     plan.n_fwd = (int)work.size();
     plan.n_bwd = (int)bwork.size();
@@ -282,6 +297,12 @@ int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const f
     a.dv = dv;
     a.status = status;
     a.st = st;
+    if (plan->zero_end > plan->zero_begin) {
+        const size_t pitch = (size_t)L * kHeadDim * sizeof(bf16), width = (size_t)(plan->zero_end - plan->zero_begin) * kHeadDim * sizeof(bf16);
+        if (cudaMemset2DAsync(dk + (size_t)plan->zero_begin * kHeadDim, pitch, 0, width, BH, stream) != cudaSuccess ||
+            cudaMemset2DAsync(dv + (size_t)plan->zero_begin * kHeadDim, pitch, 0, width, BH, stream) != cudaSuccess)
+            return HMAR_ERR_CUDA;
+    }
     return launch_bwd_tc(mq, mk, mv, mdo, macc, a, out, dout, dq, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 

@@ -214,14 +214,15 @@ def test_fp32_debug_build_512_shape_one_head():
     _run_training(_Wl(CONFIGS["512_d24_train"].side_lens, B=1, H=1), torch.float32)
 
 
-WINDOWS = [("causal", hmar.HMAR_WINDOW_CAUSAL), ("self", hmar.HMAR_WINDOW_SELF)]
+WINDOWS = [("causal", hmar.HMAR_WINDOW_CAUSAL), ("self", hmar.HMAR_WINDOW_SELF), ("prev", hmar.HMAR_WINDOW_PREV)]
 
 
 @pytest.mark.parametrize("window", WINDOWS, ids=[w[0] for w in WINDOWS])
-@pytest.mark.parametrize("sides", [(1, 2, 3, 4), (3, 11), (12, 11, 1), (2, 1, 3, 1, 2), (1, 2, 3, 4, 5, 6, 8, 10, 13, 16), (16, 3, 17)])
+@pytest.mark.parametrize("sides", [(1, 2, 3, 4), (3, 11), (12, 11, 1), (2, 1, 3, 1, 2), (1, 2, 3, 4, 5, 6, 8, 10, 13, 16), (16, 3, 17), (5,), (1, 1), (9, 13, 18)])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_other_block_masks_fwd_bwd(sides, dtype, window):
-    """VAR's block-causal mask and the block-diagonal mask through the *_window entry points."""
+    """VAR's block-causal mask, the block-diagonal mask and the preceding-scale mask (whose last scale's keys have
+    no queries: dK = dV = 0 there) through the *_window entry points."""
     wl = _Wl(sides)
     is_f32 = dtype == torch.float32
     q, k, v, do = training_inputs(wl, bf16=not is_f32)
@@ -232,9 +233,18 @@ def test_other_block_masks_fwd_bwd(sides, dtype, window):
     _assert_lse(lse, ref_lse, is_f32)
     dq, dk, dv = hmar.hmar_attn_bwd(tq, tk, tv, out, lse, tdo, wl.side_lens, wl.softmax_scale, window=window[1])
     rq, rk, rv = orc.attn_bwd(q, k, v, do, wl.side_lens, wl.softmax_scale, window=window[0])
-    _assert_close("dq", dq, rq, is_f32)
-    _assert_close("dk", dk, rk, is_f32)
-    _assert_close("dv", dv, rv, is_f32)
+    # Under the narrow masks a one-token scale is the only key of every query of the next scale: P = 1 for all of
+    # them, and that key's dK, dV are plain sums over those queries, several times larger than O(1).  A bf16
+    # result cannot be closer than its unit roundoff 2^-8 |x|, so where the oracle's largest entry exceeds
+    # 2e-2 / 2^-8 = 5.1 the absolute limits grow in proportion (factor 1 otherwise, and always 1 for fp32).
+    def mag(ref):
+        return 1.0 if is_f32 else max(1.0, float(np.abs(ref).max()) * 2.0 ** -8 / BF16_MAX)
+    _assert_close("dq", dq, rq, is_f32, mag(rq))
+    _assert_close("dk", dk, rk, is_f32, mag(rk))
+    _assert_close("dv", dv, rv, is_f32, mag(rv))
+    if window[0] == "prev" and len(sides) > 1:
+        n_last = sides[-1] ** 2                        # nobody looks at the last scale's keys: exact zeros
+        assert not dk[:, :, -n_last:].any() and not dv[:, :, -n_last:].any()
     _no_device_error()
 
 

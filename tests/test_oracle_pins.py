@@ -97,6 +97,8 @@ def test_window_masks_pair_counts_closed_forms():
         start = np.concatenate([[0], np.cumsum(n)])
         assert orc.count_pairs(sides, "causal") == sum(n[k] * start[k + 1] for k in range(len(n)))
         assert orc.count_pairs(sides, "self") == sum(x * x for x in n)
+        # preceding scale only: n_k * n_{k-1} pairs per scale, and the first scale on itself
+        assert orc.count_pairs(sides, "prev") == n[0] * n[0] + sum(n[k] * n[k - 1] for k in range(1, len(n)))
     # densities quoted for the paper's shapes: block-causal 61.9 % at L = 680 and 65.2 % at L = 2240
     assert orc.count_pairs(CONFIGS["256_d16_fwd"].side_lens, "causal") / 680 ** 2 == pytest.approx(0.619, abs=5e-4)
     assert orc.count_pairs(CONFIGS["512_d24_train"].side_lens, "causal") / 2240 ** 2 == pytest.approx(0.652, abs=5e-4)
@@ -105,12 +107,64 @@ def test_window_masks_pair_counts_closed_forms():
 
 
 def test_window_masks_single_scale_all_dense_and_nesting():
-    for w in ("markov", "causal", "self"):
+    for w in ("markov", "causal", "self", "prev"):
         assert orc.window_mask((5,), w).all()
     sides = (2, 3, 1, 4)
     S, M, C = (orc.window_mask(sides, w) for w in ("self", "markov", "causal"))
     assert not (S & ~M).any() and not (M & ~C).any() and S.sum() < M.sum() < C.sum()
     assert (S == S.T).all() and not (C == C.T).all()
+    # the preceding-scale mask and the block-diagonal one split the Markov mask between them, except for the
+    # first scale's own block, which both hold
+    P = orc.window_mask(sides, "prev")
+    assert ((P | S) == M).all() and (P & S).sum() == sides[0] ** 4
+    assert P.any(axis=1).all()                                           # no empty row
+    assert not P[:, -(sides[-1] ** 2):].any()                            # nobody looks at the last scale's keys
+
+
+def test_prev_window_literals_and_locality():
+    # sides (1, 1, 2): token 0 sees itself; token 1 sees token 0; tokens 2-5 see token 1 only
+    expect = np.zeros((6, 6), dtype=bool)
+    expect[0, 0] = expect[1, 0] = True
+    expect[2:, 1] = True
+    assert (orc.window_mask((1, 1, 2), "prev") == expect).all()
+    rng = np.random.default_rng(21)
+    sides = (2, 1, 3, 2)
+    n = [x * x for x in sides]
+    start = np.concatenate([[0], np.cumsum(n)])
+    L = int(start[-1])
+    q, k, v, do = (rng.standard_normal((L, 6)) for _ in range(4))
+    out, lse = orc.attn_fwd(q, k, v, sides, 0.4, window="prev")
+    # scale 2 (one token in scale 1... a single key) : rows of scale index 2 see the single token of scale index 1,
+    # so their output is exactly that token's value and lse is the one logit
+    np.testing.assert_allclose(out[start[2]:start[3]], np.broadcast_to(v[start[1]], (n[2], 6)), rtol=1e-13)
+    np.testing.assert_allclose(lse[start[2]:start[3]], 0.4 * q[start[2]:start[3]] @ k[start[1]], rtol=1e-13)
+    # rows of scale k do not move when their own scale's keys change, and do when the preceding scale's do
+    k2, v2 = k.copy(), v.copy()
+    k2[start[3]:] += 1.0
+    v2[start[3]:] -= 2.0
+    out2, _ = orc.attn_fwd(q, k2, v2, sides, 0.4, window="prev")
+    assert np.array_equal(out, out2)                                     # the last scale's keys reach nothing
+    v3 = v.copy()
+    v3[start[2]:start[3]] += 1.0
+    out3, _ = orc.attn_fwd(q, k, v3, sides, 0.4, window="prev")
+    assert np.array_equal(out[:start[3]], out3[:start[3]]) and not np.allclose(out[start[3]:], out3[start[3]:])
+    # the last scale is plain dense attention over the preceding scale's keys (library softmax as the check)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q[start[3]:])[None], torch.from_numpy(k[start[2]:start[3]])[None],
+        torch.from_numpy(v[start[2]:start[3]])[None], scale=0.4)[0].numpy()
+    np.testing.assert_allclose(out[start[3]:], ref, rtol=1e-12, atol=1e-12)
+    # backward: keys of the last scale get exactly zero, and central differences agree elsewhere
+    dq, dk, dv = orc.attn_bwd(q, k, v, do, sides, 0.4, window="prev")
+    assert not dk[start[3]:].any() and not dv[start[3]:].any()
+    for grad, idx in ((dq, 0), (dk, 1), (dv, 2)):
+        for _ in range(12):
+            i, d = int(rng.integers(L)), int(rng.integers(6))
+            args = [q.copy(), k.copy(), v.copy()]
+            args[idx][i, d] += 1e-6
+            fp = (orc.attn_fwd(*args, sides, 0.4, window="prev")[0] * do).sum()
+            args[idx][i, d] -= 2e-6
+            fm = (orc.attn_fwd(*args, sides, 0.4, window="prev")[0] * do).sum()
+            assert (fp - fm) / 2e-6 == pytest.approx(grad[i, d], rel=1e-6, abs=1e-8)
 
 
 def test_self_window_is_independent_attention_per_scale():
