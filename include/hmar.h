@@ -183,6 +183,21 @@ int hmar_attn_scale_step_strided(const void* q, const void* k_prev, const void* 
                                  long long kv_cur_head_stride, long long out_head_stride,
                                  float softmax_scale, void* stream);
 
+/* The sampler's step next to the attention at inference (Alg. 2, "Multi-scale VQ-VAE Reconstruction", lines
+ * 7-8: x~_k = interpolate(lookup(V, r_k), H_K, W_K), x~_{1:k} = x~_{1:k-1} + x~_k) fused with the token
+ * selection of a masked refinement sub-step (Sec. 4.2: the positions in the sub-step's mask take the newly
+ * generated token, the others keep theirs).  The paper does not name the interpolation; this is bicubic
+ * convolution with a = -0.75, half-pixel sample positions and border-clamped indices.
+ *   xhat       : [B, C, out_side, out_side] fp32, device, updated in place (+= the interpolated codes)
+ *   codebook   : [V, C] fp32, device
+ *   tokens_new : [B, side, side] int32 ids, device;  tokens_old : the same shape, or NULL when mask is NULL
+ *   mask       : [B, side, side] bytes, nonzero = take tokens_new there; NULL = take tokens_new everywhere
+ *   tokens_out : [B, side, side] int32 or NULL; receives the selected map (must not alias the inputs)
+ * side <= out_side <= 4096.  Ids outside [0, V) are clamped.  One kernel, asynchronous on `stream`. */
+int hmar_recon_accumulate(float* xhat, const float* codebook, const int* tokens_old, const int* tokens_new,
+                          const unsigned char* mask, int* tokens_out, int B, int C, int V, int side, int out_side,
+                          void* stream);
+
 /* Host-side scale-block scheduler (Sec. 4.1: the kernel visits only the live blocks of the mask).
  * Writes the work list of one head for `direction` 0 = forward (tiles of query rows, each with the
  * contiguous key range it must visit) or 1 = backward (tiles of key rows with their query range).
@@ -198,8 +213,20 @@ int hmar_schedule_tiles_window(int n_scales, const int* side_lens, int window, i
 
 /* Blocks until the work queued on the current device has finished, then returns the code recorded
  * by the kernels since the last call (HMAR_OK, or HMAR_ERR_DEVICE_TIMEOUT with *detail, if not NULL,
- * telling which wait gave up) and clears it.  Diagnostics only; never needed for correct results. */
+ * telling which wait gave up) and clears it.
+ * Every wait inside the tensor-core kernels is bounded (about one second of wall time, which on a GPU shared
+ * by time slicing includes the time the context is switched out).  When one runs out, the block gives up,
+ * the word latches, and every tensor-core kernel launched on the device afterwards returns at once WITHOUT
+ * writing its outputs, while the entry points keep returning HMAR_OK (they never synchronise).  A caller
+ * that must know whether its results are valid therefore calls this function after the work it cares
+ * about: HMAR_OK means every kernel since the previous call ran to completion. */
 int hmar_device_status(int* detail);
+
+/* Self-test of that mechanism (no counterpart in the paper): launches one block that waits, through the
+ * kernels' own wait routine with a limit of one millisecond, on a barrier nothing ever arrives on.  The wait
+ * gives up and the block returns; the next hmar_device_status() reports HMAR_ERR_DEVICE_TIMEOUT with detail
+ * 0xD1A6 and clears it.  Nothing traps or faults; the context stays usable. */
+int hmar_selftest_bounded_wait(void* stream);
 
 /* Per-kernel timing for benchmarks.  Between hmar_profile_begin() and hmar_profile_end() every kernel
  * the library launches is bracketed by two CUDA events on its stream.  hmar_profile_end() synchronises

@@ -167,3 +167,61 @@ def scale_step(q, k_prev, v_prev, k_cur, v_cur, softmax_scale):
     M = np.ones((q.shape[-2], kk.shape[-2]), dtype=bool)
     P, lse = attention_probs(q, kk, M, softmax_scale)
     return P @ vv, lse
+
+
+# ----------------------------------------------------------------------------------------------
+# The sampler's steps on either side of the attention at inference (Alg. 2, "Multi-scale VQ-VAE
+# Reconstruction"; Sec. 4.2, the masked refinement sub-steps).  The paper writes
+#     x~_k = interpolate(lookup(V, r_k), H_K, W_K),   x~_{1:k} = x~_{1:k-1} + x~_k
+# and, inside a scale, regenerates only the positions chosen by the sub-step's mask.  It does not say
+# which interpolation; reading used here: bicubic convolution with the kernel parameter a = -0.75 and
+# half-pixel sample positions, source indices clamped at the border (what the VAR tokenizer family that
+# HMAR builds on uses to bring a coarse token map to the final resolution).
+
+def select_tokens(tokens_old, tokens_new, mask):
+    """Sec. 4.2: positions where `mask` is nonzero take the newly generated token, the others keep theirs."""
+    return np.where(np.asarray(mask) != 0, np.asarray(tokens_new), np.asarray(tokens_old))
+
+
+def _cubic_weights(t, a=-0.75):
+    """Weights of the four taps at offsets -1, 0, 1, 2 for a sample at fractional position t in [0, 1)."""
+    def near(x):      # |x| <= 1
+        return ((a + 2.0) * x - (a + 3.0)) * x * x + 1.0
+
+    def far(x):       # 1 < |x| < 2
+        return ((a * x - 5.0 * a) * x + 8.0 * a) * x - 4.0 * a
+    return np.array([far(t + 1.0), near(t), near(1.0 - t), far(2.0 - t)])
+
+
+def bicubic_upsample(x, out_side):
+    """x: [..., h, w] float64 -> [..., out_side, out_side], plain loops over the output pixels."""
+    x = np.asarray(x, dtype=np.float64)
+    h, w = x.shape[-2], x.shape[-1]
+    out = np.zeros(x.shape[:-2] + (out_side, out_side), dtype=np.float64)
+    for oy in range(out_side):
+        sy = (oy + 0.5) * h / out_side - 0.5
+        iy = int(np.floor(sy))
+        wy = _cubic_weights(sy - iy)
+        for ox in range(out_side):
+            sx = (ox + 0.5) * w / out_side - 0.5
+            ix = int(np.floor(sx))
+            wx = _cubic_weights(sx - ix)
+            acc = 0.0
+            for a in range(4):
+                yy = min(max(iy - 1 + a, 0), h - 1)
+                for b in range(4):
+                    xx = min(max(ix - 1 + b, 0), w - 1)
+                    acc = acc + wy[a] * wx[b] * x[..., yy, xx]
+            out[..., oy, ox] = acc
+    return out
+
+
+def recon_accumulate(xhat, codebook, tokens, out_side):
+    """One pass of Alg. 2's loop body: xhat [B, C, out_side, out_side] + interpolate(lookup(codebook, tokens)).
+
+    codebook: [V, C]; tokens: [B, side, side] integer ids.  Returns the new running reconstruction (float64)."""
+    codebook = np.asarray(codebook, dtype=np.float64)
+    tokens = np.asarray(tokens)
+    looked = codebook[tokens]                                   # [B, side, side, C]
+    coarse = np.moveaxis(looked, -1, 1)                         # [B, C, side, side]
+    return np.asarray(xhat, dtype=np.float64) + bicubic_upsample(coarse, out_side)

@@ -30,7 +30,7 @@ EXPORTED_SYMBOLS = (
     "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_fwd_window", "hmar_attn_fwd_window_f32", "hmar_attn_fwd_packed",
     "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd", "hmar_attn_bwd_f32", "hmar_attn_bwd_window",
     "hmar_attn_bwd_window_f32", "hmar_schedule_tiles_window", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_attn_scale_step_strided", "hmar_schedule_tiles",
-    "hmar_device_status", "hmar_profile_begin", "hmar_profile_end", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
+    "hmar_recon_accumulate", "hmar_device_status", "hmar_selftest_bounded_wait", "hmar_profile_begin", "hmar_profile_end", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
     "hmar_status_string",
 )
 
@@ -70,7 +70,9 @@ def lib():
     ll = ctypes.c_longlong
     L.hmar_attn_scale_step_strided.argtypes = [vp] * 7 + [i, i, i, i, i, ll, ll, ll, ll, fp, vp]
     L.hmar_schedule_tiles.argtypes = [i, ip, i, ctypes.POINTER(ctypes.c_int32), i]
+    L.hmar_recon_accumulate.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
     L.hmar_device_status.argtypes = [ip]
+    L.hmar_selftest_bounded_wait.argtypes = [vp]
     L.hmar_profile_begin.restype = None
     L.hmar_profile_end.argtypes = [ctypes.c_char_p, ctypes.c_size_t]
     L.hmar_debug_force_simt.argtypes = [i]
@@ -254,6 +256,22 @@ def hmar_attn_scale_step_strided(q, k_prev, v_prev, k_cur, v_cur, side_prev, sid
     return out, lse
 
 
+def hmar_recon_accumulate(xhat, codebook, tokens_new, tokens_old=None, mask=None, tokens_out=None, stream=None):
+    """xhat [B,C,S,S] fp32 += bicubic(lookup(codebook [V,C], selected tokens [B,s,s])); returns xhat.
+    `mask` (uint8 [B,s,s]) chooses tokens_new over tokens_old per position; `tokens_out` receives the selection."""
+    _need(xhat, codebook, tokens_new, tokens_old, mask, tokens_out)
+    if xhat.dtype != torch.float32 or codebook.dtype != torch.float32 or tokens_new.dtype != torch.int32:
+        raise TypeError("xhat and codebook must be float32, tokens int32")
+    if mask is not None and mask.dtype != torch.uint8:
+        raise TypeError("mask must be uint8")
+    B, C, S, _ = xhat.shape
+    V = codebook.shape[0]
+    side = tokens_new.shape[1]
+    _check(lib().hmar_recon_accumulate(_ptr(xhat), _ptr(codebook), _ptr(tokens_old), _ptr(tokens_new), _ptr(mask),
+                                       _ptr(tokens_out), B, C, V, side, S, _stream(stream)), "hmar_recon_accumulate")
+    return xhat
+
+
 def hmar_schedule_tiles(side_lens, direction, window=HMAR_WINDOW_MARKOV):
     """Work list of one head as a list of dicts (host only; needs no GPU)."""
     sides, n = _sides(side_lens)
@@ -271,6 +289,11 @@ def hmar_device_status():
     detail = ctypes.c_int(0)
     status = lib().hmar_device_status(ctypes.byref(detail))
     return status, detail.value
+
+
+def hmar_selftest_bounded_wait(stream=None):
+    """Launches the one-block kernel whose bounded wait must run out (see include/hmar.h)."""
+    _check(lib().hmar_selftest_bounded_wait(_stream(stream)), "hmar_selftest_bounded_wait")
 
 
 def hmar_profile_begin():

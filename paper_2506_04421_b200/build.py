@@ -7,7 +7,7 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libhmar.so")
-SOURCES = ["api.cu", "schedule.cpp", "simt_kernels.cu", "tc_dispatch.cu", "fwd_sm100.cu", "bwd_sm100.cu", "noalloc_bwd.cu", "step_small.cu"]
+SOURCES = ["api.cu", "schedule.cpp", "simt_kernels.cu", "tc_dispatch.cu", "fwd_sm100.cu", "bwd_sm100.cu", "noalloc_bwd.cu", "step_small.cu", "recon.cu"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

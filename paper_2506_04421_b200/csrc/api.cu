@@ -13,6 +13,7 @@
 
 #include "hmar_common.h"
 #include "launchers.h"
+#include "tc_common.h"
 #include "tc_launchers.h"
 
 namespace hmar {
@@ -378,6 +379,28 @@ int hmar_profile_end(char* report, size_t capacity) {
         report[n] = 0;
     }
     return HMAR_OK;
+}
+
+int hmar_recon_accumulate(float* xhat, const float* codebook, const int* tokens_old, const int* tokens_new,
+                          const unsigned char* mask, int* tokens_out, int B, int C, int V, int side, int out_side,
+                          void* stream) {
+    if (B <= 0 || C <= 0 || V <= 0 || side <= 0 || out_side <= 0 || side > 4096 || out_side > 4096 || C > 4096) return HMAR_ERR_BAD_ARG;
+    if (side > out_side) return HMAR_ERR_BAD_ARG;                       // the step only ever enlarges a token map
+    if (xhat == nullptr || codebook == nullptr || tokens_new == nullptr) return HMAR_ERR_BAD_ARG;
+    if (mask != nullptr && tokens_old == nullptr) return HMAR_ERR_BAD_ARG;
+    if (tokens_out != nullptr && (tokens_out == tokens_new || tokens_out == tokens_old)) return HMAR_ERR_BAD_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return HMAR_ERR_CUDA; }
+    return launch_recon_accumulate(xhat, codebook, tokens_old, tokens_new, mask, tokens_out, B, C, V, side, out_side,
+                                   static_cast<cudaStream_t>(stream)) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
+}
+
+int hmar_selftest_bounded_wait(void* stream) {
+    int rc = check_device();
+    if (rc != HMAR_OK) return rc;
+    int* status = device_status_ptr();
+    if (status == nullptr) return HMAR_ERR_CUDA;
+    return launch_selftest_wait(status, static_cast<cudaStream_t>(stream)) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
 int hmar_debug_force_simt(int enable) { return g_force_simt.exchange(enable ? 1 : 0); }

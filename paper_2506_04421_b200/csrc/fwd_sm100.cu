@@ -436,7 +436,29 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     }
 }
 
+// Self-test of the bounded waits: one block waits on a barrier that nothing ever arrives on, with a limit of
+// one millisecond, through the very wait and report functions the kernels use.  The wait gives up, the block
+// records HMAR_ERR_DEVICE_TIMEOUT with location 0xD1A6 in the status word and returns; nothing traps.
+__global__ void hmar_selftest_wait_kernel(int* status) {
+    __shared__ uint64_t never;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(&never, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    const bool ok = __all_sync(0xffffffffu, mbar_wait(&never, 0, &abort_flag, 1000000ull));
+    if (!ok && threadIdx.x == 0) report_timeout(status, 0xD1A6);
+}
+
 }  // namespace
+
+cudaError_t launch_selftest_wait(int* status, cudaStream_t stream) {
+    hmar_selftest_wait_kernel<<<1, 32, 0, stream>>>(status);
+    count_launch(1);
+    return cudaGetLastError();
+}
 
 size_t fwd_tc_smem_bytes() { return sizeof(SharedStorage) + 1024; }
 

@@ -31,4 +31,8 @@ cudaError_t simt_bwd(const T* q, const T* k, const T* v, const T* out, const flo
                      T* dq, T* dk, T* dv, float* delta, int BH, const ScaleTable& st, float scale,
                      cudaStream_t stream);
 
+cudaError_t launch_recon_accumulate(float* xhat, const float* codebook, const int* tokens_old, const int* tokens_new,
+                                    const unsigned char* mask, int* tokens_out, int B, int C, int V, int side, int out_side,
+                                    cudaStream_t stream);
+
 }  // namespace hmar

@@ -1,0 +1,91 @@
+// The sampler's step next to the attention at inference: the running multi-scale reconstruction
+// (paper Alg. 2, "Multi-scale VQ-VAE Reconstruction": x~_k = interpolate(lookup(V, r_k), H_K, W_K),
+// x~_{1:k} = x~_{1:k-1} + x~_k) fused with the token selection of a masked refinement sub-step (Sec. 4.2:
+// only the positions in the sub-step's mask take the newly generated token).
+//
+// One pass does, per output pixel of the final resolution: select the 4 x 4 neighbourhood's token ids
+// (new where the mask is set, old elsewhere), look their code vectors up, interpolate bicubically
+// (a = -0.75, half-pixel sample positions, border indices clamped) and add the result to the running
+// reconstruction in place.  The reconstruction is read and written exactly once (the algorithmic HBM bytes
+// of the step); the codebook (V x C fp32, 512 KB for V = 4096, C = 32) and the token maps stay in L2 / L1.
+// A thread owns one output pixel and walks the channels, so a warp's accesses to the [B, C, H, W] tensor
+// are 128-byte rows for every channel.
+#include <cuda_runtime.h>
+
+#include "hmar_common.h"
+#include "launchers.h"
+
+namespace hmar {
+namespace {
+
+__device__ __forceinline__ void cubic_weights(float t, float (&w)[4]) {
+    const float a = -0.75f;
+    const float x0 = t + 1.f, x1 = t, x2 = 1.f - t, x3 = 2.f - t;
+    w[0] = ((a * x0 - 5.f * a) * x0 + 8.f * a) * x0 - 4.f * a;
+    w[1] = ((a + 2.f) * x1 - (a + 3.f)) * x1 * x1 + 1.f;
+    w[2] = ((a + 2.f) * x2 - (a + 3.f)) * x2 * x2 + 1.f;
+    w[3] = ((a * x3 - 5.f * a) * x3 + 8.f * a) * x3 - 4.f * a;
+}
+
+__global__ void __launch_bounds__(256)
+hmar_recon_accumulate_kernel(float* __restrict__ xhat, const float* __restrict__ codebook,
+                             const int* __restrict__ tokens_old, const int* __restrict__ tokens_new,
+                             const unsigned char* __restrict__ mask, int* __restrict__ tokens_out,
+                             int B, int C, int V, int side, int out_side) {
+    const long long pix = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long n_pix = (long long)B * out_side * out_side;
+    // the selected token map is also written back (one thread per coarse position), for the next sub-step
+    if (tokens_out != nullptr && pix < (long long)B * side * side) {
+        const int keep = (mask == nullptr || mask[pix] != 0) ? tokens_new[pix] : tokens_old[pix];
+        tokens_out[pix] = keep;
+    }
+    if (pix >= n_pix) return;
+    const int ox = (int)(pix % out_side), oy = (int)((pix / out_side) % out_side), b = (int)(pix / ((long long)out_side * out_side));
+    const float ratio = (float)side / (float)out_side;
+    const float sy = (oy + 0.5f) * ratio - 0.5f, sx = (ox + 0.5f) * ratio - 0.5f;
+    const int iy = (int)floorf(sy), ix = (int)floorf(sx);
+    float wy[4], wx[4];
+    cubic_weights(sy - (float)iy, wy);
+    cubic_weights(sx - (float)ix, wx);
+    // ids of the 16 neighbours, selected, clamped into the codebook (an id outside [0, V) reads code 0 or V - 1)
+    int id[16];
+    float wgt[16];
+#pragma unroll
+    for (int a = 0; a < 4; ++a) {
+        const int yy = min(max(iy - 1 + a, 0), side - 1);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int xx = min(max(ix - 1 + c, 0), side - 1);
+            const long long pos = ((long long)b * side + yy) * side + xx;
+            int t = (mask == nullptr || mask[pos] != 0) ? tokens_new[pos] : tokens_old[pos];
+            id[a * 4 + c] = min(max(t, 0), V - 1);
+            wgt[a * 4 + c] = wy[a] * wx[c];
+        }
+    }
+    float* dst = xhat + ((long long)b * C) * out_side * out_side + (long long)oy * out_side + ox;
+    const long long plane = (long long)out_side * out_side;
+    for (int ch = 0; ch < C; ++ch) {
+        float acc = 0.f;
+#pragma unroll
+        for (int n = 0; n < 16; ++n) acc = fmaf(wgt[n], __ldg(codebook + (long long)id[n] * C + ch), acc);
+        dst[ch * plane] += acc;
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_recon_accumulate(float* xhat, const float* codebook, const int* tokens_old, const int* tokens_new,
+                                    const unsigned char* mask, int* tokens_out, int B, int C, int V, int side, int out_side,
+                                    cudaStream_t stream) {
+    const long long n_pix = (long long)B * out_side * out_side;
+    const unsigned grid = (unsigned)((n_pix + 255) / 256);
+    {
+        KernelTimer timer("hmar_recon_accumulate_kernel", stream);
+        hmar_recon_accumulate_kernel<<<grid, 256, 0, stream>>>(xhat, codebook, tokens_old, tokens_new, mask, tokens_out, B, C, V,
+                                                              side, out_side);
+    }
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+}  // namespace hmar

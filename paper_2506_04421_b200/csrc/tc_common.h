@@ -73,6 +73,7 @@ struct BwdArgs {
 };
 
 size_t fwd_tc_smem_bytes();
+cudaError_t launch_selftest_wait(int* status, cudaStream_t stream);
 cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& dout_map,
                           const CUtensorMap& dq_acc_map, const BwdArgs& args, const __nv_bfloat16* out, const __nv_bfloat16* dout,
                           __nv_bfloat16* dq, int BH, cudaStream_t stream);

@@ -76,6 +76,15 @@ def _assert_bf16_dq(name, dq, ref, bound, max_factor=1.0):
     assert mx <= BF16_MAX * max_factor and mean <= BF16_MEAN * max_factor, msg
 
 
+def _guarded(shape, dtype, guards, pad=512):
+    """An output tensor with `pad` canary elements before and after it in the same allocation; appends to
+    `guards` a function that says whether the canaries are still intact."""
+    n = int(np.prod(shape))
+    flat = torch.full((n + 2 * pad,), 77.0, dtype=dtype, device="cuda")
+    guards.append(lambda: bool((flat[:pad] == 77.0).all() and (flat[pad + n:] == 77.0).all()))
+    return flat[pad:pad + n].view(*shape)
+
+
 def _no_device_error():
     status, detail = hmar.hmar_device_status()
     assert status == hmar.HMAR_OK, f"device status {status} detail {detail:#x}"
@@ -98,12 +107,16 @@ def _run_training(wl, dtype, gain=1.0, backward=True, simt=False):
     prev = hmar.hmar_debug_force_simt(simt)
     try:
         tq, tk, tv, tdo = (to_device(x, wl.B, wl.H, dtype) for x in (q, k, v, do))
-        out, lse = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale)
+        # every output sits between canary stretches that the kernels must leave alone
+        guards = []
+        out, lse = _guarded(tq.shape, dtype, guards), _guarded(tq.shape[:3], torch.float32, guards)
+        hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale, out=out, lse=lse)
         ref_out, ref_lse = orc.attn_fwd(q, k, v, wl.side_lens, wl.softmax_scale)
         _assert_close("out", out, ref_out, is_f32)
         _assert_lse(lse, ref_lse, is_f32)
         if backward:
-            dq, dk, dv = hmar.hmar_attn_bwd(tq, tk, tv, out, lse, tdo, wl.side_lens, wl.softmax_scale)
+            dq, dk, dv = (_guarded(tq.shape, dtype, guards) for _ in range(3))
+            hmar.hmar_attn_bwd(tq, tk, tv, out, lse, tdo, wl.side_lens, wl.softmax_scale, dq=dq, dk=dk, dv=dv)
             rq, rk, rv = orc.attn_bwd(q, k, v, do, wl.side_lens, wl.softmax_scale)
             if is_f32 or gain == 1.0:
                 _assert_close("dq", dq, rq, is_f32, mag_k)
@@ -112,6 +125,7 @@ def _run_training(wl, dtype, gain=1.0, backward=True, simt=False):
             _assert_close("dk", dk, rk, is_f32, mag_k)
             _assert_close("dv", dv, rv, is_f32)
         _no_device_error()
+        assert all(intact() for intact in guards), "a kernel wrote outside its output tensor"
     finally:
         hmar.hmar_debug_force_simt(prev)
 
@@ -464,6 +478,26 @@ def test_scale_step_matches_training_forward_rows():
         assert (l - lse[:, :, cur]).abs().max().item() <= 1e-4
 
 
+def test_bounded_wait_runs_out_reports_and_leaves_the_context_usable():
+    """A kernel whose bounded wait runs out (a barrier nothing arrives on, 1 ms limit, the kernels' own wait
+    and report routines) returns by itself; the status word reports it once; while the word is latched the
+    tensor-core kernels return without writing; after the poll everything works again."""
+    hmar.hmar_device_status()                                   # clear whatever earlier tests left
+    hmar.hmar_selftest_bounded_wait()
+    assert hmar.hmar_device_status() == (hmar.HMAR_ERR_DEVICE_TIMEOUT, 0xD1A6)
+    assert hmar.hmar_device_status() == (hmar.HMAR_OK, 0)       # reported once, then clear
+    wl = _Wl((3, 11, 5))
+    q, k, v, do = training_inputs(wl, bf16=True)
+    tq, tk, tv, tdo = (to_device(x, wl.B, wl.H, torch.bfloat16) for x in (q, k, v, do))
+    hmar.hmar_selftest_bounded_wait()
+    out = torch.full_like(tq, 7.0)
+    hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale, out=out)      # launched while the word is latched
+    torch.cuda.synchronize()
+    assert (out == 7.0).all()
+    assert hmar.hmar_device_status()[0] == hmar.HMAR_ERR_DEVICE_TIMEOUT
+    _run_training(wl, torch.bfloat16)                           # and the library is back to normal
+
+
 def test_bad_workspace_is_rejected():
     wl = CONFIGS["tiny"]
     q, k, v, do = training_inputs(wl)
@@ -487,3 +521,29 @@ def test_repeat_calls_are_stable():
     assert torch.equal(g1[1], g2[1]) and torch.equal(g1[2], g2[2])        # dk, dv deterministic
     assert (g1[0].float() - g2[0].float()).abs().max().item() <= 2e-2     # dq: atomics, order may differ
     assert hmar.hmar_launch_count() > 0
+
+
+@pytest.mark.parametrize("side,out_side,B,C,V", [(1, 32, 3, 32, 4096), (6, 32, 2, 32, 4096), (13, 32, 2, 32, 4096), (32, 32, 2, 32, 4096),
+                                                  (3, 7, 2, 5, 17), (16, 16, 65, 32, 4096)])
+@pytest.mark.parametrize("masked", [False, True])
+def test_recon_accumulate_matches_oracle(side, out_side, B, C, V, masked):
+    """The sampler's neighbour step (Alg. 2 lines 7-8 with the sub-step's token selection, Sec. 4.2) on a synthetic
+    codebook: fp32 on the GPU against the fp64 oracle, and the selected token map bit for bit."""
+    rng = np.random.default_rng(1000 * side + out_side + int(masked))
+    codebook = rng.standard_normal((V, C)).astype(np.float32)
+    old = rng.integers(0, V, (B, side, side)).astype(np.int32)
+    new = rng.integers(0, V, (B, side, side)).astype(np.int32)
+    mask = rng.integers(0, 2, (B, side, side)).astype(np.uint8)
+    x0 = rng.standard_normal((B, C, out_side, out_side)).astype(np.float32)
+    dev = lambda a: torch.from_numpy(a).cuda()
+    guards = []
+    xhat = _guarded(x0.shape, torch.float32, guards)
+    xhat.copy_(dev(x0))
+    t_out = torch.full((B, side, side), -1, dtype=torch.int32, device="cuda")
+    hmar.hmar_recon_accumulate(xhat, dev(codebook), dev(new), dev(old) if masked else None, dev(mask) if masked else None, t_out)
+    sel = orc.select_tokens(old, new, mask) if masked else new
+    ref = orc.recon_accumulate(x0, codebook, sel, out_side)
+    assert torch.equal(t_out.cpu(), torch.from_numpy(sel.astype(np.int32)))
+    err = np.abs(xhat.double().cpu().numpy() - ref)
+    assert err.max() <= 1e-5 * max(1.0, np.abs(ref).max()), f"max abs err {err.max():.3e}"
+    assert all(intact() for intact in guards)

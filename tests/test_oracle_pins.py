@@ -521,3 +521,64 @@ def test_pins_detect_planted_mistakes(monkeypatch):
     # (7) dQ and dK swapped
     monkeypatch.setattr(orc, "attn_bwd", lambda *a: (good_bwd(*a)[1], good_bwd(*a)[0], good_bwd(*a)[2]))
     assert fails(test_backward_finite_differences)
+
+
+# --------------------------------------------------------------------------- the sampler's neighbour step (Alg. 2)
+
+def test_cubic_weights_literals_and_partition_of_unity():
+    # a = -0.75: at t = 0 the sample sits on a source pixel; at t = 1/2 the classic (-3, 19, 19, -3) / 32 taps
+    np.testing.assert_allclose(orc._cubic_weights(0.0), [0.0, 1.0, 0.0, 0.0], atol=1e-15)
+    np.testing.assert_allclose(orc._cubic_weights(0.5), np.array([-3.0, 19.0, 19.0, -3.0]) / 32.0, atol=1e-15)
+    for t in np.linspace(0.0, 0.999, 37):
+        w = orc._cubic_weights(t)
+        assert w.sum() == pytest.approx(1.0, abs=1e-14)
+        np.testing.assert_allclose(w[::-1], orc._cubic_weights(1.0 - t) if t > 0 else [0, 0, 1, 0], atol=1e-14)
+
+
+def test_bicubic_upsample_against_the_library_routine_and_special_cases():
+    rng = np.random.default_rng(31)
+    for h, H in ((1, 8), (2, 7), (3, 8), (5, 16), (13, 32), (6, 6)):
+        x = rng.standard_normal((2, 3, h, h))
+        ref = torch.nn.functional.interpolate(torch.from_numpy(x), size=(H, H), mode="bicubic", align_corners=False).numpy()
+        np.testing.assert_allclose(orc.bicubic_upsample(x, H), ref, rtol=1e-12, atol=1e-13)
+    x = rng.standard_normal((4, 4))
+    assert np.array_equal(orc.bicubic_upsample(x, 4), x)                               # same size: identity
+    np.testing.assert_allclose(orc.bicubic_upsample(np.full((3, 3), 2.5), 9), 2.5, rtol=1e-14)   # constants stay
+    np.testing.assert_allclose(orc.bicubic_upsample(np.array([[1.75]]), 5), 1.75, rtol=1e-14)    # one token: flat image
+    y = rng.standard_normal((4, 4))
+    np.testing.assert_allclose(orc.bicubic_upsample(2.0 * x - 3.0 * y, 11),
+                               2.0 * orc.bicubic_upsample(x, 11) - 3.0 * orc.bicubic_upsample(y, 11), rtol=1e-12, atol=1e-13)
+    # transposing the input transposes the output (rows and columns are treated alike)
+    np.testing.assert_allclose(orc.bicubic_upsample(x.T, 10), orc.bicubic_upsample(x, 10).T, rtol=1e-13, atol=1e-14)
+
+
+def test_select_tokens_and_recon_accumulate():
+    rng = np.random.default_rng(32)
+    B, C, V, side, S = 2, 5, 17, 3, 8
+    codebook = rng.standard_normal((V, C))
+    old, new = rng.integers(0, V, (B, side, side)), rng.integers(0, V, (B, side, side))
+    mask = rng.integers(0, 2, (B, side, side))
+    sel = orc.select_tokens(old, new, mask)
+    assert np.array_equal(sel[mask == 1], new[mask == 1]) and np.array_equal(sel[mask == 0], old[mask == 0])
+    assert np.array_equal(orc.select_tokens(old, new, np.zeros_like(mask)), old)
+    assert np.array_equal(orc.select_tokens(old, new, np.ones_like(mask)), new)
+    x0 = rng.standard_normal((B, C, S, S))
+    x1 = orc.recon_accumulate(x0, codebook, sel, S)
+    # written out by hand for one output pixel and channel: the 16 taps around the sample position
+    b, c, oy, ox = 1, 3, 5, 2
+    sy, sx = (oy + 0.5) * side / S - 0.5, (ox + 0.5) * side / S - 0.5
+    iy, ix = int(np.floor(sy)), int(np.floor(sx))
+    wy, wx = orc._cubic_weights(sy - iy), orc._cubic_weights(sx - ix)
+    acc = 0.0
+    for a in range(4):
+        for d in range(4):
+            yy, xx = min(max(iy - 1 + a, 0), side - 1), min(max(ix - 1 + d, 0), side - 1)
+            acc += wy[a] * wx[d] * codebook[sel[b, yy, xx], c]
+    assert x1[b, c, oy, ox] == pytest.approx(x0[b, c, oy, ox] + acc, rel=1e-13)
+    # a codebook of one repeated vector: every pixel gains exactly that vector, whatever the tokens
+    flat = np.tile(rng.standard_normal((1, C)), (V, 1))
+    np.testing.assert_allclose(orc.recon_accumulate(x0, flat, sel, S) - x0, flat[0][None, :, None, None] * np.ones((B, C, S, S)), rtol=1e-12, atol=1e-13)
+    # Alg. 2's loop: the reconstruction after two scales is the sum of the two interpolated maps
+    t2 = rng.integers(0, V, (B, 5, 5))
+    both = orc.recon_accumulate(orc.recon_accumulate(np.zeros((B, C, S, S)), codebook, sel, S), codebook, t2, S)
+    np.testing.assert_allclose(both, orc.recon_accumulate(np.zeros((B, C, S, S)), codebook, t2, S) + (x1 - x0), rtol=1e-12, atol=1e-13)
