@@ -498,28 +498,57 @@ def run_ours(args, wl):
     h_out, h_dq, h_dk, h_dv = (torch.empty_like(hq).pin_memory() for _ in range(4))
     h_lse = torch.empty((B, H, L), dtype=torch.float32).pin_memory()
 
+    # The batch is cut into chunks; chunk c is copied in on one stream, computed on a second and copied out on a
+    # third, so the host-to-device copies, the kernels and the device-to-host copies of different chunks overlap
+    # (PCIe carries both directions at once).  Every call goes through the C ABI on the chunk's own slices.
+    n_chunks = 4 if B % 4 == 0 else 1
+    cb = B // n_chunks
+    s_in, s_run, s_out = (torch.cuda.Stream(device=dev) for _ in range(3))
+    ws_c = [torch.empty(hmar.hmar_attn_bwd_workspace_bytes(cb, H, D, sides), dtype=torch.uint8, device=dev) for _ in range(2)]
+    ev_in = [torch.cuda.Event() for _ in range(n_chunks)]
+    ev_run = [torch.cuda.Event() for _ in range(n_chunks)]
+    ev_free = [torch.cuda.Event() for _ in range(n_chunks)]     # the chunk's results have left the device
+
     def e2e_step():
-        q.copy_(hq, non_blocking=True)
-        k.copy_(hk, non_blocking=True)
-        v.copy_(hv, non_blocking=True)
-        do.copy_(hdo, non_blocking=True)
-        step()
-        h_out.copy_(out, non_blocking=True)
-        h_lse.copy_(lse, non_blocking=True)
-        h_dq.copy_(dq, non_blocking=True)
-        h_dk.copy_(dk, non_blocking=True)
-        h_dv.copy_(dv, non_blocking=True)
+        for c in range(n_chunks):
+            sl = slice(c * cb, (c + 1) * cb)
+            with torch.cuda.stream(s_in):
+                for d_t, h_t in ((q, hq), (k, hk), (v, hv), (do, hdo)):
+                    d_t[sl].copy_(h_t[sl], non_blocking=True)
+                ev_in[c].record(s_in)
+            with torch.cuda.stream(s_run):
+                s_run.wait_event(ev_in[c])
+                if c >= 2:
+                    s_run.wait_event(ev_free[c - 2])           # the workspace of chunk c - 2 is reused
+                hmar.hmar_attn_fwd(q[sl], k[sl], v[sl], sides, scale, out=out[sl], lse=lse[sl], stream=s_run)
+                hmar.hmar_attn_bwd(q[sl], k[sl], v[sl], out[sl], lse[sl], do[sl], sides, scale, dq=dq[sl], dk=dk[sl], dv=dv[sl],
+                                   workspace=ws_c[c % 2], stream=s_run)
+                ev_run[c].record(s_run)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_run[c])
+                for h_t, d_t in ((h_out, out), (h_lse, lse), (h_dq, dq), (h_dk, dk), (h_dv, dv)):
+                    h_t[sl].copy_(d_t[sl], non_blocking=True)
+                ev_free[c].record(s_out)
+        cur = torch.cuda.current_stream()
+        cur.wait_stream(s_out)
+        cur.wait_stream(s_run)
+        cur.wait_stream(s_in)
 
     e2e_steps = max(2, min(args.steps, 5))
     e2e_step()
     barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for st_ in (s_in, s_run, s_out):
+        st_.wait_stream(torch.cuda.current_stream())
     e0.record()
     for _ in range(e2e_steps):
+        for st_ in (s_in, s_run, s_out):
+            st_.wait_stream(torch.cuda.current_stream())      # a step starts after the previous one has ended
         e2e_step()
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
+    args.e2e_note = f"{n_chunks} batch chunks on three streams (copy in, compute, copy out), pinned host buffers"
     return _finish(args, wl, world, rank, dev, total_ms, e2e_ms, fwd_ms, bwd_ms, launches, clocks, kernels)
 
 
@@ -570,7 +599,8 @@ def _finish(args, wl, world, rank, dev, total_ms, e2e_ms, fwd_ms, bwd_ms, launch
             "kernels": per_kernel,
             "cpu_baseline": cpu_base,
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms,
-                    "h2d_bytes_per_step": 4 * elem, "d2h_bytes_per_step": 4 * elem + 4 * B * H * L},
+                    "h2d_bytes_per_step": 4 * elem, "d2h_bytes_per_step": 4 * elem + 4 * B * H * L,
+                    "how": getattr(args, "e2e_note", "")},
             "gpu_launches": int(launches),
             "clocks": clocks,
         }

@@ -7,7 +7,7 @@
 //   logits ready -> softmax warpgroup -> P ready -> tensor core (O += P V, next logits) -> ...
 // A chain spends most of its time waiting for the other side (the round trip through the barriers and the
 // tensor core's queue is longer than either side's work), so what keeps an SM busy is the number of
-// independent chains on it: a block is kept small (192 threads, 128 TMEM columns, 50 KB of shared memory)
+// independent chains on it: a block is kept small (256 threads, 128 TMEM columns, 50 KB of shared memory)
 // and FOUR blocks share an SM.  Each block's set-up, first copies and epilogue, during which it computes
 // nothing, are then overlapped by three running chains instead of being a quarter of its life.
 //   warps 0-3   softmax: one query row per thread, 64 logits per tile read from TMEM once; the running
@@ -21,9 +21,12 @@
 //   warp 5      issues tcgen05.mma: S = Q K^T (both operands in shared memory), O += P V (P from TMEM, V an
 //               MN-major shared-memory operand), one burst per tile: O += P V of tile j, then S of tile
 //               j + 1 into the columns P has just left
+//   warps 6-7   idle: setmaxnreg works on whole warpgroups (four warps), so the producer and the MMA warp
+//               sit in a full second warpgroup (a block of 192 threads cannot redistribute its registers;
+//               without the redistribution the softmax warps spill and the kernel is 4 % slower)
 // TMEM columns: S/P [0,64), O [64,128).
-// Registers: the block starts with 80 per thread (four blocks per SM); the softmax warps raise theirs to
-// 96 and the other two warps drop to 48 (setmaxnreg), the same total.
+// Registers: the block starts with 64 per thread (four blocks per SM); the softmax warpgroup raises its
+// to 88 and the second warpgroup drops to 40 (setmaxnreg), the same total.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -44,11 +47,11 @@ constexpr int D = kHeadDim;
 constexpr int NSTAGE = 2;
 constexpr int Q_BYTES = BM * D * 2;             // 16 KB
 constexpr int TILE_BYTES = BN * D * 2;          // 8 KB
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 256;
 constexpr int NUM_SOFTMAX_THREADS = 128;
 constexpr int PRODUCER_WARP = 4, MMA_WARP = 5;
-constexpr int REGS_START = 80, REGS_SOFTMAX = 96, REGS_MISC = 48;
-static_assert(4 * REGS_SOFTMAX + 2 * REGS_MISC == 6 * REGS_START, "register budget of the block");
+constexpr int REGS_START = 64, REGS_SOFTMAX = 88, REGS_MISC = 40;
+static_assert(4 * REGS_SOFTMAX + 4 * REGS_MISC == 8 * REGS_START, "register budget of the block");
 constexpr uint32_t TMEM_COLS = 128;
 constexpr uint32_t COL_S = 0, COL_O = 64;
 constexpr float kRescaleThreshold = 8.0f;       // in log2 units
@@ -167,6 +170,7 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
     volatile int* abort_flag = &sm.abort_flag;
 
     if (warp >= PRODUCER_WARP) {
+        reg_dec<REGS_MISC>();
         if (warp == PRODUCER_WARP) {
             // ================================================================== TMA producer
             // The whole warp runs the control flow; one elected lane issues the copies (a warp that has split
@@ -203,7 +207,7 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 const uint64_t t0 = globaltimer_ns();
                 while (globaltimer_ns() - t0 < 2000000ull) { }
             }
-        } else {
+        } else if (warp == MMA_WARP) {
             // ================================================================== MMA issuer
             // The whole warp runs the control flow; one elected lane issues.  Descriptors are built once and
             // advanced by adding (byte offset >> 4), so issuing an MMA costs a few instructions.
@@ -286,6 +290,7 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         }
     } else {
         // ================================================================== softmax warps + epilogue
+        reg_inc<REGS_SOFTMAX>();
         const int r = warp * 32 + lane;                        // row inside the tile
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
         const int row = w.row_begin + r;
