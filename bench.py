@@ -328,30 +328,40 @@ def time_training_shape(hmar, wl_x, dev, window, reps=3):
     return f_ms, b_ms
 
 
-def time_packed_forward(hmar, wl_x, dev, reps=5):
-    """ms of the forward on the packed projection output [B,L,3,H,D] -> [B,L,H,D], and of the copies that the
-    contiguous entry point would need around it for the same data (context leg)."""
+def time_packed_step(hmar, wl_x, dev, reps=5):
+    """ms of forward and backward on the packed projection layouts (qkv, dqkv [B,L,3,H,D]; out, dout [B,L,H,D]), and
+    of the transposing copies that the contiguous entry points would need around them for the same data: three in
+    and one out for the forward, one more in (dout) and three out (dq, dk, dv) for the backward (context leg)."""
     import torch
     from workloads.device import bulk_normal
     B, H, L, D = wl_x.B, wl_x.H, wl_x.L, wl_x.D
     qkv = bulk_normal(wl_x.seed, 9, B, L, 3 * H, D, torch.bfloat16, dev).view(B, L, 3, H, D)
+    dout = bulk_normal(wl_x.seed, 10, B, L, H, D, torch.bfloat16, dev)
     out = torch.empty((B, L, H, D), dtype=torch.bfloat16, device=dev)
     lse = torch.empty((B, H, L), dtype=torch.float32, device=dev)
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
-    p_ms = c_ms = 0.0
+    dqkv = torch.empty_like(qkv)
+    ws = torch.empty(hmar.hmar_attn_bwd_workspace_bytes(B, H, D, wl_x.side_lens), dtype=torch.uint8, device=dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+    f_ms = b_ms = c_ms = 0.0
     for it in range(reps + 1):
         ev[0].record()
         hmar.hmar_attn_fwd_packed(qkv, wl_x.side_lens, wl_x.softmax_scale, out=out, lse=lse)
         ev[1].record()
-        q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3).contiguous() for i in range(3))
-        o = torch.empty_like(q)
-        o.permute(0, 2, 1, 3).contiguous()
+        hmar.hmar_attn_bwd_packed(qkv, out, lse, dout, wl_x.side_lens, wl_x.softmax_scale, dqkv=dqkv, workspace=ws)
         ev[2].record()
+        q, k, v = (qkv[:, :, i].permute(0, 2, 1, 3).contiguous() for i in range(3))
+        do_c = dout.permute(0, 2, 1, 3).contiguous()
+        q.permute(0, 2, 1, 3).contiguous()                  # out back to [B,L,H,D]
+        for i in range(3):
+            dqkv[:, :, i].copy_(q.permute(0, 2, 1, 3))      # dq, dk, dv into the packed gradient
+        ev[3].record()
         torch.cuda.synchronize()
+        del q, k, v, do_c
         if it:
-            p_ms += ev[0].elapsed_time(ev[1]) / reps
-            c_ms += ev[1].elapsed_time(ev[2]) / reps
-    return p_ms, c_ms
+            f_ms += ev[0].elapsed_time(ev[1]) / reps
+            b_ms += ev[1].elapsed_time(ev[2]) / reps
+            c_ms += ev[2].elapsed_time(ev[3]) / reps
+    return f_ms, b_ms, c_ms
 
 
 def run_reference(args, wl):
@@ -477,9 +487,10 @@ def run_ours(args, wl):
                                                    "markov_speedup_bwd": round(cb / bwd_ms, 3)}
             torch.cuda.empty_cache()
             # forward on the packed QKV projection output, and the transposing copies it makes unnecessary
-            pk, cp = time_packed_forward(hmar, wl, dev)
-            extras["packed_qkv_forward"] = {"fwd_ms": round(pk, 4), "transposes_avoided_ms": round(cp, 4),
-                                            "layout": "qkv [B,L,3,H,D] -> out [B,L,H,D]"}
+            pf, pb, cp = time_packed_step(hmar, wl, dev)
+            extras["packed_qkv_step"] = {"fwd_ms": round(pf, 4), "bwd_ms": round(pb, 4), "contiguous_fwd_ms": round(fwd_ms, 4),
+                                         "contiguous_bwd_ms": round(bwd_ms, 4), "transposes_avoided_ms": round(cp, 4),
+                                         "layout": "qkv, dqkv [B,L,3,H,D]; out, dout [B,L,H,D]"}
             torch.cuda.empty_cache()
             # 1024 x 1024 (synthetic 14-scale schedule ending at 64 x 64, L = 9451), Markov mask
             wl_big = CONFIGS["1024_d24_train"]

@@ -76,8 +76,7 @@ int hmar_attn_fwd_f32(const float* q, const float* k, const float* v, float* out
  * transformer block's QKV projection and its output projection; reading the projection's layout saves the
  * transposing copies around the kernel).  bf16 only, Markovian mask.
  *   qkv : [B,L,3,H,D] in (q, k, v of a token side by side);  out : [B,L,H,D] out (the layout the output
- *   projection reads);  lse : [B,H,L] fp32 out, as for hmar_attn_fwd (the backward takes contiguous
- *   [B,H,L,D] tensors only).  All pointers device, 16-byte aligned.  HMAR_ERR_UNSUPPORTED while the
+ *   projection reads);  lse : [B,H,L] fp32 out, as for hmar_attn_fwd.  All pointers device, 16-byte aligned.  HMAR_ERR_UNSUPPORTED while the
  *   fall-back kernels are forced (they read contiguous tensors only); other errors as for hmar_attn_fwd. */
 int hmar_attn_fwd_packed(const void* qkv, void* out, float* lse, int B, int H, int D, int n_scales,
                          const int* side_lens, float softmax_scale, void* stream);
@@ -91,6 +90,16 @@ int hmar_attn_fwd_window(const void* q, const void* k, const void* v, void* out,
 int hmar_attn_fwd_window_f32(const float* q, const float* k, const float* v, float* out, float* lse,
                              int B, int H, int D, int n_scales, const int* side_lens, int window,
                              float softmax_scale, void* stream);
+
+/* Training backward on the packed layouts of hmar_attn_fwd_packed, so that a training step needs no
+ * transposing copy on either side of the attention (Sec. 4.1).  bf16 only, Markovian mask.
+ *   qkv : [B,L,3,H,D] in;  out, dout : [B,L,H,D] in;  lse : [B,H,L] in (from hmar_attn_fwd_packed);
+ *   dqkv : [B,L,3,H,D] out (dq, dk, dv of a token side by side, the layout the projection's backward reads).
+ *   workspace : as for hmar_attn_bwd (same size).  Same arithmetic as hmar_attn_bwd: dk and dv carry the very
+ *   bits the contiguous entry point gives for the same values.  Errors as for hmar_attn_fwd_packed. */
+int hmar_attn_bwd_packed(const void* qkv, const void* out, const float* lse, const void* dout, void* dqkv,
+                         void* workspace, size_t workspace_bytes, int B, int H, int D, int n_scales,
+                         const int* side_lens, float softmax_scale, void* stream);
 
 /* Bytes of caller-provided device scratch the backward needs for this problem (0 on bad arguments).
  * The scratch holds delta = rowsum(dO o O) and the fp32 dQ accumulator; its contents on entry do not

@@ -27,7 +27,7 @@ HMAR_WINDOW_SELF = 2        # scale k only (block-diagonal)
 HMAR_WINDOW_PREV = 3        # scale k-1 only; the first scale attends to itself
 
 EXPORTED_SYMBOLS = (
-    "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_fwd_window", "hmar_attn_fwd_window_f32", "hmar_attn_fwd_packed",
+    "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_fwd_window", "hmar_attn_fwd_window_f32", "hmar_attn_fwd_packed", "hmar_attn_bwd_packed",
     "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd", "hmar_attn_bwd_f32", "hmar_attn_bwd_window",
     "hmar_attn_bwd_window_f32", "hmar_schedule_tiles_window", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_attn_scale_step_strided", "hmar_schedule_tiles",
     "hmar_recon_accumulate", "hmar_device_status", "hmar_selftest_bounded_wait", "hmar_profile_begin", "hmar_profile_end", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
@@ -57,6 +57,7 @@ def lib():
     L.hmar_attn_fwd_window.argtypes = [vp, vp, vp, vp, vp, i, i, i, i, ip, i, fp, vp]
     L.hmar_attn_fwd_window_f32.argtypes = L.hmar_attn_fwd_window.argtypes
     L.hmar_attn_fwd_packed.argtypes = [vp, vp, vp, i, i, i, i, ip, fp, vp]
+    L.hmar_attn_bwd_packed.argtypes = [vp] * 5 + [vp, ctypes.c_size_t, i, i, i, i, ip, fp, vp]
     L.hmar_attn_bwd_workspace_bytes.argtypes = [i, i, i, i, ip]
     L.hmar_attn_bwd_workspace_bytes.restype = ctypes.c_size_t
     L.hmar_attn_bwd.argtypes = [vp] * 9 + [vp, ctypes.c_size_t, i, i, i, i, ip, fp, vp]
@@ -160,6 +161,23 @@ def hmar_attn_fwd_packed(qkv, side_lens, softmax_scale, out=None, lse=None, stre
     _check(lib().hmar_attn_fwd_packed(_ptr(qkv), _ptr(out), _ptr(lse), B, H, D, n, sides, float(softmax_scale),
                                       _stream(stream)), "hmar_attn_fwd_packed")
     return out, lse
+
+
+def hmar_attn_bwd_packed(qkv, out, lse, dout, side_lens, softmax_scale, dqkv=None, workspace=None, stream=None):
+    """Training backward on the packed layouts. qkv [B,L,3,H,D], out and dout [B,L,H,D], lse [B,H,L].
+    Returns dqkv [B,L,3,H,D]."""
+    _need(qkv, out, lse, dout, dqkv, workspace)
+    B, L, three, H, D = qkv.shape
+    if three != 3 or _is_f32(qkv):
+        raise ValueError("qkv must be bfloat16 [B, L, 3, H, D]")
+    dqkv = torch.empty_like(qkv) if dqkv is None else dqkv
+    if workspace is None:
+        workspace = torch.empty(hmar_attn_bwd_workspace_bytes(B, H, D, side_lens), dtype=torch.uint8, device=qkv.device)
+    sides, n = _sides(side_lens)
+    _check(lib().hmar_attn_bwd_packed(_ptr(qkv), _ptr(out), _ptr(lse), _ptr(dout), _ptr(dqkv), _ptr(workspace),
+                                      workspace.numel(), B, H, D, n, sides, float(softmax_scale), _stream(stream)),
+           "hmar_attn_bwd_packed")
+    return dqkv
 
 
 def hmar_attn_bwd_workspace_bytes(B, H, D, side_lens):

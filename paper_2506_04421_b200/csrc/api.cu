@@ -239,6 +239,31 @@ int hmar_attn_fwd_packed(const void* qkv, void* out, float* lse, int B, int H, i
                          static_cast<cudaStream_t>(stream));
 }
 
+int hmar_attn_bwd_packed(const void* qkv, const void* out, const float* lse, const void* dout, void* dqkv,
+                         void* workspace, size_t workspace_bytes, int B, int H, int D, int n_scales,
+                         const int* side_lens, float softmax_scale, void* stream) {
+    int rc = check_shape(B, H, D);
+    if (rc != HMAR_OK) return rc;
+    ScaleTable st;
+    rc = check_sides(n_scales, side_lens, HMAR_WINDOW_MARKOV, &st);
+    if (rc != HMAR_OK) return rc;
+    if (check_scale(softmax_scale) != HMAR_OK) return HMAR_ERR_BAD_ARG;
+    const void* ptrs[] = {qkv, out, lse, dout, dqkv};
+    for (const void* p : ptrs)
+        if (p == nullptr || !aligned16(p)) return HMAR_ERR_BAD_ARG;
+    if (workspace == nullptr || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0 ||
+        workspace_bytes < hmar_attn_bwd_workspace_bytes(B, H, D, n_scales, side_lens))
+        return HMAR_ERR_WORKSPACE;
+    rc = check_device();
+    if (rc != HMAR_OK) return rc;
+    if (g_force_simt.load()) return HMAR_ERR_UNSUPPORTED;      // the fall-back kernels read contiguous tensors only
+    const int L = st.start[st.n_scales];
+    float* delta = static_cast<float*>(workspace);
+    float* dq_acc = reinterpret_cast<float*>(static_cast<char*>(workspace) + round256((size_t)B * H * L * sizeof(float)));
+    return tc_bwd_packed((const bf16*)qkv, (const bf16*)out, lse, (const bf16*)dout, (bf16*)dqkv, delta, dq_acc, B, H, st,
+                         softmax_scale, device_status_ptr(), static_cast<cudaStream_t>(stream));
+}
+
 int hmar_attn_fwd(const void* q, const void* k, const void* v, void* out, float* lse, int B, int H, int D,
                   int n_scales, const int* side_lens, float softmax_scale, void* stream) {
     return hmar_attn_fwd_window(q, k, v, out, lse, B, H, D, n_scales, side_lens, HMAR_WINDOW_MARKOV, softmax_scale, stream);

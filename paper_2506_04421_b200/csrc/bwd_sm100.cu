@@ -209,7 +209,10 @@ __device__ __forceinline__ int first_item_at_cost(const BwdArgs& args, long long
 
 // CHUNKED: the block's items are several runs (long sequences, see the launcher); otherwise one contiguous run,
 // and the item loops compile to plain counting.
-template <bool CHUNKED>
+// STRIDED: the bf16 tensors have the strides given in the arguments (packed projection layouts); otherwise they are
+// dense [BH, L, 64] and every address is formed with compile-time strides (the dense instantiation is the one the
+// benchmarks run: the extra address arithmetic and code of the strided one cost it a tenth of its speed).
+template <bool CHUNKED, bool STRIDED>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
@@ -325,6 +328,7 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             for (int item = 0; item < n_items && ok; ++item) {
                 const int g = item_at(item, run);
                 const int bh = g / n_work;
+                const int batch = STRIDED ? bh / args.heads_per_batch : 0, head = STRIDED ? bh - batch * args.heads_per_batch : bh;
                 const BwdWork w = get_work(g);
                 const int n_steps = steps_of(w);
                 if (item >= 2) {
@@ -334,9 +338,9 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                 }
                 if (leader) {
                     mbar_arrive_expect_tx(&sm.k_full[item & 1], TILE_BYTES);
-                    tma_load_3d(sm.k[item & 1], &map_k, &sm.k_full[item & 1], 0, w.row_begin, bh);
+                    tma_load_4d(sm.k[item & 1], &map_k, &sm.k_full[item & 1], 0, w.row_begin, head, batch);
                     // the V rows are read by the drain warps a few steps from now: bring them into L2
-                    tma_prefetch_3d(&map_v, 0, w.row_begin, bh);
+                    tma_prefetch_4d(&map_v, 0, w.row_begin, head, batch);
                 }
                 __syncwarp();
                 for (int i = 0; i < n_steps; ++i, ++gs) {
@@ -348,8 +352,8 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     }
                     if (leader) {
                         mbar_arrive_expect_tx(&sm.qdo_full[slot], 2 * TILE_BYTES);
-                        tma_load_3d(sm.q[slot], &map_q, &sm.qdo_full[slot], 0, q0, bh);
-                        tma_load_3d(sm.dout[slot], &map_do, &sm.qdo_full[slot], 0, q0, bh);
+                        tma_load_4d(sm.q[slot], &map_q, &sm.qdo_full[slot], 0, q0, head, batch);
+                        tma_load_4d(sm.dout[slot], &map_do, &sm.qdo_full[slot], 0, q0, head, batch);
                     }
                     __syncwarp();
                 }
@@ -578,7 +582,13 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         auto copy_kv = [&](int gc, int item, bool wait_free) -> bool {
             const BwdWork wc = get_work(gc);
             const int row = wc.row_begin + r;
-            const uint4* vsrc = reinterpret_cast<const uint4*>(args.v + ((size_t)(gc / n_work) * L + row) * D);
+            const uint4* vsrc;
+            if (STRIDED) {
+                const int cbh = gc / n_work, cb = cbh / args.heads_per_batch, ch = cbh - cb * args.heads_per_batch;
+                vsrc = reinterpret_cast<const uint4*>(args.v + cb * args.in_batch + ch * args.in_head + (long long)row * args.in_row);
+            } else {
+                vsrc = reinterpret_cast<const uint4*>(args.v + ((size_t)(gc / n_work) * L + row) * D);
+            }
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
                 const uint4 val = row < L ? __ldg(vsrc + c) : make_uint4(0u, 0u, 0u, 0u);
@@ -634,7 +644,14 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         if (r < w.row_count) {
                             const float mul = part < 2 ? args.softmax_scale : 1.f;
                             __nv_bfloat16* base = part < 2 ? args.dk : args.dv;
-                            uint4* dst = reinterpret_cast<uint4*>(base + ((size_t)bh * L + w.row_begin + r) * D + (part & 1) * 32);
+                            uint4* dst;
+                            if (STRIDED) {
+                                const int ob = bh / args.heads_per_batch, oh = bh - ob * args.heads_per_batch;
+                                dst = reinterpret_cast<uint4*>(base + ob * args.g_batch + oh * args.g_head +
+                                                               (long long)(w.row_begin + r) * args.g_row + (part & 1) * 32);
+                            } else {
+                                dst = reinterpret_cast<uint4*>(base + ((size_t)bh * L + w.row_begin + r) * D + (part & 1) * 32);
+                            }
 #pragma unroll
                             for (int t = 0; t < 4; ++t) {
                                 uint4 o;
@@ -768,11 +785,25 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 }
 
 // ------------------------------------------------------------------------------------------------
+// Offset (elements) of row `row` (= bh * L + l) of a strided bf16 tensor.
+struct RowLayout {
+    int L, heads_per_batch;
+    long long row, head, batch;
+    template <bool STRIDED>
+    __device__ __forceinline__ long long offset(size_t r) const {
+        if (!STRIDED) return (long long)r * D;
+        const int bh = (int)(r / (size_t)L), l = (int)(r - (size_t)bh * L);
+        const int b = bh / heads_per_batch, h = bh - b * heads_per_batch;
+        return b * batch + h * head + l * row;
+    }
+};
+
 // delta_i = sum_d dO_id * O_id  (one warp per 4 rows: 8 lanes x 16 bytes cover a row).  The same pass
 // clears the fp32 dQ accumulator (32 bytes per lane), which saves a separate pass over it.
+template <bool STRIDED>
 __global__ void __launch_bounds__(256)
 hmar_bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
-                      float* __restrict__ delta, float* __restrict__ dq_acc, size_t n_rows) {
+                      float* __restrict__ delta, float* __restrict__ dq_acc, size_t n_rows, const RowLayout lay) {
     const size_t row = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 3;
     const int part = threadIdx.x & 7;
     float acc = 0.f;
@@ -780,8 +811,9 @@ hmar_bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16
         float4* z = reinterpret_cast<float4*>(dq_acc + row * D + part * 8);
         z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
         z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
-        const uint4 a = *reinterpret_cast<const uint4*>(out + row * D + part * 8);
-        const uint4 b = *reinterpret_cast<const uint4*>(dout + row * D + part * 8);
+        const long long off = lay.template offset<STRIDED>(row) + part * 8;
+        const uint4 a = *reinterpret_cast<const uint4*>(out + off);
+        const uint4 b = *reinterpret_cast<const uint4*>(dout + off);
         const __nv_bfloat162* pa = reinterpret_cast<const __nv_bfloat162*>(&a);
         const __nv_bfloat162* pb = reinterpret_cast<const __nv_bfloat162*>(&b);
 #pragma unroll
@@ -798,8 +830,10 @@ hmar_bwd_delta_kernel(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16
 }
 
 // dq = bf16(scale * dq_acc)
+template <bool STRIDED>
 __global__ void __launch_bounds__(256)
-hmar_bwd_dq_convert_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, float scale, size_t n8) {
+hmar_bwd_dq_convert_kernel(const float* __restrict__ acc, __nv_bfloat16* __restrict__ dq, float scale, size_t n8,
+                           const RowLayout lay) {
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= n8) return;
     const float4 a = reinterpret_cast<const float4*>(acc)[2 * idx];
@@ -809,7 +843,7 @@ hmar_bwd_dq_convert_kernel(const float* __restrict__ acc, __nv_bfloat16* __restr
     o.y = pack_bf16(a.z * scale, a.w * scale);
     o.z = pack_bf16(b.x * scale, b.y * scale);
     o.w = pack_bf16(b.z * scale, b.w * scale);
-    reinterpret_cast<uint4*>(dq)[idx] = o;
+    *reinterpret_cast<uint4*>(dq + lay.template offset<STRIDED>(idx >> 3) + (idx & 7) * 8) = o;
 }
 
 }  // namespace
@@ -827,18 +861,20 @@ static int sm_count() {
     return cached[dev];
 }
 
-cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& dout_map,
-                          const CUtensorMap& dq_acc_map, const BwdArgs& args, const __nv_bfloat16* out, const __nv_bfloat16* dout,
-                          __nv_bfloat16* dq, int BH, cudaStream_t stream) {
+template <bool STRIDED>
+static cudaError_t launch_bwd_tc_layout(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& dout_map,
+                                        const CUtensorMap& dq_acc_map, const BwdArgs& args, const __nv_bfloat16* out,
+                                        const __nv_bfloat16* dout, __nv_bfloat16* dq, int BH, cudaStream_t stream) {
     const size_t smem = sizeof(SharedStorage) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<false, STRIDED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<true, STRIDED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const size_t n_rows = (size_t)BH * args.L;
     {
         KernelTimer timer("hmar_bwd_delta_kernel", stream);
-        hmar_bwd_delta_kernel<<<(unsigned)((n_rows * 8 + 255) / 256), 256, 0, stream>>>(out, dout, args.delta_w, args.dq_acc, n_rows);
+        const RowLayout lay{args.L, args.heads_per_batch, args.od_row, args.od_head, args.od_batch};
+        hmar_bwd_delta_kernel<STRIDED><<<(unsigned)((n_rows * 8 + 255) / 256), 256, 0, stream>>>(out, dout, args.delta_w, args.dq_acc, n_rows, lay);
     }
     {
         KernelTimer timer("hmar_bwd_tc_kernel", stream);
@@ -854,17 +890,31 @@ cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUte
             while (a.split > 0 && ((long long)BH * a.split + grid - 1) / grid > MAX_CHUNKS) a.split >>= 1;
         }
         if (a.split > 0)
-            hmar_bwd_tc_kernel<true><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
+            hmar_bwd_tc_kernel<true, STRIDED><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
         else
-            hmar_bwd_tc_kernel<false><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
+            hmar_bwd_tc_kernel<false, STRIDED><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
     }
     const size_t n8 = n_rows * D / 8;
     {
         KernelTimer timer("hmar_bwd_dq_convert_kernel", stream);
-        hmar_bwd_dq_convert_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, stream>>>(args.dq_acc, dq, args.softmax_scale, n8);
+        const RowLayout lay{args.L, args.heads_per_batch, args.g_row, args.g_head, args.g_batch};
+        hmar_bwd_dq_convert_kernel<STRIDED><<<(unsigned)((n8 + 255) / 256), 256, 0, stream>>>(args.dq_acc, dq, args.softmax_scale, n8, lay);
     }
     count_launch(3);
     return cudaGetLastError();
+}
+
+cudaError_t launch_bwd_tc(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& dout_map,
+                          const CUtensorMap& dq_acc_map, const BwdArgs& args, const __nv_bfloat16* out, const __nv_bfloat16* dout,
+                          __nv_bfloat16* dq, int BH, cudaStream_t stream) {
+    // dense [BH, L, 64] everywhere: the instantiation with compile-time strides
+    const long long row = D, head = (long long)args.L * D;
+    const bool dense = args.in_row == row && args.od_row == row && args.g_row == row && args.in_head == head &&
+                       args.od_head == head && args.g_head == head &&
+                       (args.heads_per_batch == BH || (args.in_batch == args.heads_per_batch * head &&
+                                                       args.od_batch == args.in_batch && args.g_batch == args.in_batch));
+    return dense ? launch_bwd_tc_layout<false>(q, k, v, dout_map, dq_acc_map, args, out, dout, dq, BH, stream)
+                 : launch_bwd_tc_layout<true>(q, k, v, dout_map, dq_acc_map, args, out, dout, dq, BH, stream);
 }
 
 }  // namespace hmar

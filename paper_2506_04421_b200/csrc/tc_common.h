@@ -64,8 +64,15 @@ struct BwdArgs {
     const float* delta;      // [BH, L] rowsum(dO o O) (read by the main kernel)
     float* delta_w;          // same buffer, written by the preprocess kernel
     float* dq_acc;           // [BH, L, 64] fp32 accumulator
-    const __nv_bfloat16* k;  // [BH, L, 64] (read directly for the rows that go to TMEM)
-    const __nv_bfloat16* v;
+    // Layout of the bf16 tensors: head bh is head bh % heads_per_batch of batch bh / heads_per_batch, and element
+    // (batch, head, row, d) sits at batch * *_batch + head * *_head + row * *_row + d (strides in elements).  q, k, v
+    // share the `in` strides, out and dout the `od` strides, dq, dk, dv the `g` strides; lse, delta and the fp32 dQ
+    // accumulator are always dense [BH, L(, 64)].
+    int heads_per_batch;
+    long long in_row, in_head, in_batch;
+    long long od_row, od_head, od_batch;
+    long long g_row, g_head, g_batch;
+    const __nv_bfloat16* v;  // read directly for the rows that go to TMEM
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;
     int* status;

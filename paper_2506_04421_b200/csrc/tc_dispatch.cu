@@ -38,20 +38,6 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// Tensor map of a [heads, rows, 64] bf16 tensor read in boxes of 128 rows x 64 columns with the
-// 128-byte swizzle; rows past the end of a head read as zeros.
-static bool make_rows_map(CUtensorMap* map, const void* base, int heads, int rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (fn == nullptr) return false;
-    const cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)rows, (cuuint64_t)heads};
-    const cuuint64_t strides[2] = {(cuuint64_t)kHeadDim * 2, (cuuint64_t)rows * kHeadDim * 2};
-    const cuuint32_t box[3] = {(cuuint32_t)kHeadDim, (cuuint32_t)kTileRows, 1};
-    const cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // 4-D map (64 elements, rows, heads, batches) with the strides of the tensor in elements; boxes of `box_rows`
 // rows of one head.  Serves the contiguous [B, H, rows, 64] layout and a packed [B, rows, 3, H, 64] one alike.
 constexpr int kFwdKeyRows = 64;      // key rows per tile of the forward kernel (its query tiles are kTileRows high)
@@ -269,15 +255,21 @@ int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const b
     return launch_fwd_tc(mq, mk0, mv0, mk1, mv1, a, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
-int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const float* lse, const bf16* dout,
-           bf16* dq, bf16* dk, bf16* dv, float* delta, float* dq_acc, int BH, const ScaleTable& st, float scale,
-           int* status, cudaStream_t stream) {
+// Backward on tensors whose layout is given by strides (elements): q, k, v share one layout, out and dout another,
+// dq, dk, dv a third.
+struct Strides3 { long long row, head, batch; };
+static int tc_bwd_strided(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const float* lse, const bf16* dout,
+                          bf16* dq, bf16* dk, bf16* dv, float* delta, float* dq_acc, int B, int H, const ScaleTable& st,
+                          float scale, Strides3 in, Strides3 od, Strides3 g, int* status, cudaStream_t stream) {
     const Plan* plan = get_plan(st);
     if (plan == nullptr) return HMAR_ERR_CUDA;
     const int L = st.start[st.n_scales];
+    const int BH = B * H;
     CUtensorMap mq, mk, mv, mdo, macc;
-    if (!make_rows_map(&mq, q, BH, L) || !make_rows_map(&mk, k, BH, L) || !make_rows_map(&mv, v, BH, L) ||
-        !make_rows_map(&mdo, dout, BH, L) || !make_acc_map(&macc, dq_acc, (size_t)BH * L))
+    if (!make_rows_map4(&mq, q, B, H, L, in.row, in.head, in.batch, kTileRows) ||
+        !make_rows_map4(&mk, k, B, H, L, in.row, in.head, in.batch, kTileRows) ||
+        !make_rows_map4(&mv, v, B, H, L, in.row, in.head, in.batch, kTileRows) ||
+        !make_rows_map4(&mdo, dout, B, H, L, od.row, od.head, od.batch, kTileRows) || !make_acc_map(&macc, dq_acc, (size_t)BH * L))
         return HMAR_ERR_CUDA;
     BwdArgs a{};
     a.work = plan->bwd_work;
@@ -291,24 +283,58 @@ int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const f
     a.delta = delta;
     a.delta_w = delta;
     a.dq_acc = dq_acc;
-    a.k = k;
+    a.heads_per_batch = H;
+    a.in_row = in.row; a.in_head = in.head; a.in_batch = in.batch;
+    a.od_row = od.row; a.od_head = od.head; a.od_batch = od.batch;
+    a.g_row = g.row; a.g_head = g.head; a.g_batch = g.batch;
     a.v = v;
     a.dk = dk;
     a.dv = dv;
     a.status = status;
     a.st = st;
     if (plan->zero_end > plan->zero_begin) {
-        const size_t pitch = (size_t)L * kHeadDim * sizeof(bf16), width = (size_t)(plan->zero_end - plan->zero_begin) * kHeadDim * sizeof(bf16);
-        if (cudaMemset2DAsync(dk + (size_t)plan->zero_begin * kHeadDim, pitch, 0, width, BH, stream) != cudaSuccess ||
-            cudaMemset2DAsync(dv + (size_t)plan->zero_begin * kHeadDim, pitch, 0, width, BH, stream) != cudaSuccess)
-            return HMAR_ERR_CUDA;
+        // rows of keys that no query sees: zeros in dK and dV.  Dense heads [BH, L, 64] take one strided fill per
+        // tensor; other layouts one per head.
+        const size_t rows = (size_t)(plan->zero_end - plan->zero_begin);
+        if (g.row == kHeadDim && g.head == (long long)L * kHeadDim && (B == 1 || g.batch == (long long)H * g.head)) {
+            const size_t pitch = (size_t)L * kHeadDim * sizeof(bf16), width = rows * kHeadDim * sizeof(bf16);
+            if (cudaMemset2DAsync(dk + (size_t)plan->zero_begin * kHeadDim, pitch, 0, width, BH, stream) != cudaSuccess ||
+                cudaMemset2DAsync(dv + (size_t)plan->zero_begin * kHeadDim, pitch, 0, width, BH, stream) != cudaSuccess)
+                return HMAR_ERR_CUDA;
+        } else {
+            for (int b = 0; b < B; ++b)
+                for (int h = 0; h < H; ++h) {
+                    const long long off = b * g.batch + h * g.head + (long long)plan->zero_begin * g.row;
+                    if (cudaMemset2DAsync(dk + off, (size_t)g.row * sizeof(bf16), 0, kHeadDim * sizeof(bf16), rows, stream) != cudaSuccess ||
+                        cudaMemset2DAsync(dv + off, (size_t)g.row * sizeof(bf16), 0, kHeadDim * sizeof(bf16), rows, stream) != cudaSuccess)
+                        return HMAR_ERR_CUDA;
+                }
+        }
     }
     return launch_bwd_tc(mq, mk, mv, mdo, macc, a, out, dout, dq, BH, stream) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
+// Contiguous [B*H, L, 64] tensors: one "batch" of BH heads.
+int tc_bwd(const bf16* q, const bf16* k, const bf16* v, const bf16* out, const float* lse, const bf16* dout,
+           bf16* dq, bf16* dk, bf16* dv, float* delta, float* dq_acc, int BH, const ScaleTable& st, float scale,
+           int* status, cudaStream_t stream) {
+    const long long L = st.start[st.n_scales];
+    const Strides3 dense{kHeadDim, L * kHeadDim, (long long)BH * L * kHeadDim};
+    return tc_bwd_strided(q, k, v, out, lse, dout, dq, dk, dv, delta, dq_acc, 1, BH, st, scale, dense, dense, dense, status, stream);
+}
+
+// Packed projection layouts: qkv and dqkv [B, L, 3, H, 64], out and dout [B, L, H, 64].
+int tc_bwd_packed(const bf16* qkv, const bf16* out, const float* lse, const bf16* dout, bf16* dqkv, float* delta,
+                  float* dq_acc, int B, int H, const ScaleTable& st, float scale, int* status, cudaStream_t stream) {
+    const long long L = st.start[st.n_scales], HD = (long long)H * kHeadDim;
+    const Strides3 packed{3 * HD, kHeadDim, L * 3 * HD}, od{HD, kHeadDim, L * HD};
+    return tc_bwd_strided(qkv, qkv + HD, qkv + 2 * HD, out, lse, dout, dqkv, dqkv + HD, dqkv + 2 * HD, delta, dq_acc, B, H, st,
+                          scale, packed, od, packed, status, stream);
+}
+
 // The same tensor maps for code outside this file.
 bool make_rows_map_bf16(CUtensorMap* map, const void* base, int heads, int rows) {
-    return make_rows_map(map, base, heads, rows);
+    return make_rows_map4(map, base, 1, heads, rows, kHeadDim, (long long)rows * kHeadDim, (long long)heads * rows * kHeadDim, kTileRows);
 }
 bool make_dq_acc_map(CUtensorMap* map, const float* base, size_t rows) { return make_acc_map(map, base, rows); }
 

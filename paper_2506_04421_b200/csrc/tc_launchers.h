@@ -14,6 +14,9 @@ int tc_bwd(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* 
            const float* lse, const __nv_bfloat16* dout, __nv_bfloat16* dq, __nv_bfloat16* dk,
            __nv_bfloat16* dv, float* delta, float* dq_acc, int BH, const ScaleTable& st, float scale,
            int* status, cudaStream_t stream);
+int tc_bwd_packed(const __nv_bfloat16* qkv, const __nv_bfloat16* out, const float* lse, const __nv_bfloat16* dout,
+                  __nv_bfloat16* dqkv, float* delta, float* dq_acc, int B, int H, const ScaleTable& st, float scale,
+                  int* status, cudaStream_t stream);
 // Inference step.  Rows are 64 contiguous elements; consecutive heads of a tensor are `*_head_stride` elements apart
 // (n_rows * 64 for a dense [B,H,n,64] tensor, the ring's rows * 64 when prev and cur sit in one K/V ring buffer).
 struct StepStrides {

@@ -211,6 +211,33 @@ def test_packed_qkv_forward(sides, B, H):
     _no_device_error()
 
 
+@pytest.mark.parametrize("sides,B,H", [((1, 2, 3, 4, 6, 9, 13), 2, 3), ((3, 11), 1, 2), ((16, 3, 17), 3, 1), ((1, 2, 3, 4, 5, 6, 8, 10, 13, 16), 2, 2)])
+def test_packed_qkv_backward(sides, B, H):
+    """Backward on qkv / dqkv [B,L,3,H,D] and out / dout [B,L,H,D]: against the oracle, and dk, dv bit for bit against
+    the contiguous entry point on the same values (dq is summed in an order that varies: tolerance)."""
+    wl = _Wl(sides, B=B, H=H)
+    q, k, v, do = training_inputs(wl, bf16=True)
+    L, D = wl.L, wl.D
+    packed = np.stack([x.reshape(B, H, L, D) for x in (q, k, v)], axis=0)          # [3, B, H, L, D]
+    t = torch.from_numpy(np.ascontiguousarray(packed.transpose(1, 3, 0, 2, 4))).to(device="cuda", dtype=torch.bfloat16)
+    tdo = torch.from_numpy(np.ascontiguousarray(do.reshape(B, H, L, D).transpose(0, 2, 1, 3))).to(device="cuda", dtype=torch.bfloat16)
+    out, lse = hmar.hmar_attn_fwd_packed(t, wl.side_lens, wl.softmax_scale)
+    guards = []
+    dqkv = _guarded(t.shape, torch.bfloat16, guards)
+    hmar.hmar_attn_bwd_packed(t, out, lse, tdo, wl.side_lens, wl.softmax_scale, dqkv=dqkv)
+    refs = orc.attn_bwd(q, k, v, do, wl.side_lens, wl.softmax_scale)
+    got = [dqkv[:, :, i].permute(0, 2, 1, 3).contiguous() for i in range(3)]      # [B, H, L, D]
+    for nm, g, r in zip(("dq", "dk", "dv"), got, refs):
+        _assert_close(nm, g, r, False)
+    tq, tk, tv, tdo_c = (to_device(x, B, H, torch.bfloat16) for x in (q, k, v, do))
+    out_c, lse_c = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale)
+    dq_c, dk_c, dv_c = hmar.hmar_attn_bwd(tq, tk, tv, out_c, lse_c, tdo_c, wl.side_lens, wl.softmax_scale)
+    assert torch.equal(dk_c, got[1]) and torch.equal(dv_c, got[2])
+    assert (dq_c.float() - got[0].float()).abs().max().item() <= BF16_MAX
+    assert all(intact() for intact in guards)
+    _no_device_error()
+
+
 def test_packed_qkv_forward_full_size_matches_contiguous_bits():
     # the headline shape as bench.py's packed leg runs it: the packed entry point must give the very bits
     # of the contiguous one (which the sampled-head tests compare with the oracle at this size)
