@@ -32,7 +32,7 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
 # The captures are of the batch-4 case (traffic grows in proportion to the heads), scaled by 4 to the full batch.
-NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (231254016 + 111613440), "hmar_fwd": 4 * (82641152 + 11431936)}
+NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (234577408 + 116890624), "hmar_fwd": 4 * (82925056 + 9005056)}
 
 
 def pairs_per_head(side_lens):
@@ -621,6 +621,37 @@ def _finish(args, wl, world, rank, dev, total_ms, e2e_ms, fwd_ms, bwd_ms, launch
         dist.destroy_process_group()
 
 
+def run_case(args):
+    """A named side case run a few times (for profiling one kernel on a workload that is not the headline's):
+    `256_d30_train` = forward + backward of the L = 680 training config at its full batch; `infer_scale7` = the
+    inference step of scale 7 (169 queries, 250 keys) at B = 64, H = 24.  Prints a small JSON line."""
+    import torch
+
+    import paper_2506_04421_b200 as hmar
+    from workloads import CONFIGS
+    from workloads.device import bulk_normal
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    reps = max(1, args.steps)
+    hmar.hmar_profile_begin()
+    if args.case == "256_d30_train":
+        wl_x = CONFIGS["256_d30_train"]
+        q, k, v, do = (bulk_normal(wl_x.seed, i, wl_x.B, wl_x.H, wl_x.L, wl_x.D, torch.bfloat16, dev) for i in range(4))
+        for _ in range(args.warmup + reps):
+            out, lse = hmar.hmar_attn_fwd(q, k, v, wl_x.side_lens, wl_x.softmax_scale)
+            hmar.hmar_attn_bwd(q, k, v, out, lse, do, wl_x.side_lens, wl_x.softmax_scale)
+    else:
+        wl_x = CONFIGS["512_d24_infer"]
+        s_ = 6
+        side, sp = wl_x.side_lens[s_], wl_x.side_lens[s_ - 1]
+        t = [bulk_normal(wl_x.seed + s_, i, wl_x.B, wl_x.H, (sp if i in (1, 2) else side) ** 2, wl_x.D, torch.bfloat16, dev) for i in range(5)]
+        for _ in range(args.warmup + reps):
+            hmar.hmar_attn_scale_step(*t, sp, side, wl_x.softmax_scale, want_lse=False)
+    kern = hmar.hmar_profile_end()
+    print(json.dumps({"case": args.case, "calls": args.warmup + reps,
+                      "kernels_avg_ms": {k_: round(v_[1] / v_[0], 4) for k_, v_ in kern.items()}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -629,6 +660,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the batch size (profiling on a reduced case; named in config.workload)")
+    ap.add_argument("--case", choices=["256_d30_train", "infer_scale7"], default=None,
+                    help="run a named side case a few times instead of the benchmark (profiling)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
     ap.add_argument("--no-extras", action="store_true", help="skip the dense masked comparison and the inference sweep")
@@ -639,7 +672,9 @@ def main():
     if args.batch > 0:
         import dataclasses
         wl = dataclasses.replace(wl, B=args.batch)
-    if args.impl == "reference":
+    if args.case is not None:
+        run_case(args)
+    elif args.impl == "reference":
         run_reference(args, wl)
     else:
         run_ours(args, wl)
