@@ -271,6 +271,20 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                         ok = (rv || wait(&sm.v_full[slot], (j / NSTAGE) & 1, 0x500 + j)) &&
                              (rk || wait(&sm.k_full[slot_next], ((j + 1) / NSTAGE) & 1, 0x400 + j));
                 }
+                // The last tile of a key segment may be ragged: the rows between its last key and the next multiple of
+                // 16 (the granularity of the product over keys) belong to another scale, or to nobody.  Their P is
+                // exactly 0, but 0 x (Inf or NaN) is NaN, so these V rows are cleared before O += P V reads them:
+                // a non-finite value outside a row's window cannot reach its output.  (Whole rows: the 128-byte swizzle
+                // permutes 16-byte pieces inside a row only.)
+                if (ok) {
+                    const int n_valid = kv_tile(w, tiles0, j).n_valid;
+                    if (n_valid < n) {
+                        for (int idx = n_valid * 8 + lane; idx < n * 8; idx += 32)
+                            *reinterpret_cast<uint4*>(sm.v[slot] + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                    }
+                }
                 if (ok) ok = wait(&sm.p_full, j & 1, 0x600 + j);
                 if (!ok) break;
                 tc_fence_after();

@@ -251,6 +251,33 @@ def test_packed_qkv_forward_full_size_matches_contiguous_bits():
     _no_device_error()
 
 
+@pytest.mark.parametrize("sides", [(12, 13, 14), (13, 12, 15), (16, 13, 19, 12)])
+def test_forward_ignores_non_finite_values_outside_a_rows_window(sides):
+    """Key tiles are fetched 64 rows at a time, so the tail of a scale's last tile holds rows of the next scale.
+    Those keys are masked, but a masked P of exactly 0 times a non-finite V would still be NaN: the forward
+    clears such V rows, and a NaN logit is replaced, not scaled.  With K and V of one scale set to NaN / Inf,
+    every row that cannot see that scale must come out exactly as without them.  (Scales of at least 128 tokens:
+    a tile that packs several small scales gives its rows different windows over the same V rows, and there the
+    inputs have to be finite.)"""
+    wl = _Wl(sides)
+    q, k, v = training_inputs(wl, bf16=True, with_dout=False)
+    n = [s * s for s in wl.side_lens]
+    start = np.concatenate([[0], np.cumsum(n)])
+    tq, tk, tv = (to_device(x, wl.B, wl.H, torch.bfloat16) for x in (q, k, v))
+    clean, clean_lse = hmar.hmar_attn_fwd(tq, tk, tv, wl.side_lens, wl.softmax_scale)
+    for bad_scale in range(1, len(sides)):
+        tk2, tv2 = tk.clone(), tv.clone()
+        tk2[:, :, start[bad_scale]:start[bad_scale + 1]] = float("nan")
+        tv2[:, :, start[bad_scale]:start[bad_scale + 1]] = float("inf")
+        out, lse = hmar.hmar_attn_fwd(tq, tk2, tv2, wl.side_lens, wl.softmax_scale)
+        # rows of scales bad_scale and bad_scale + 1 see the poisoned keys; all others must be untouched
+        keep = np.ones(wl.L, dtype=bool)
+        keep[start[bad_scale]:start[min(bad_scale + 2, len(sides))]] = False
+        idx = torch.from_numpy(np.nonzero(keep)[0]).cuda()
+        assert torch.equal(out[:, :, idx], clean[:, :, idx]) and torch.equal(lse[:, :, idx], clean_lse[:, :, idx])
+    _no_device_error()
+
+
 def test_fp32_debug_build_512_shape_one_head():
     _run_training(_Wl(CONFIGS["512_d24_train"].side_lens, B=1, H=1), torch.float32)
 
