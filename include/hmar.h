@@ -44,7 +44,8 @@ typedef enum {
     HMAR_ERR_UNSUPPORTED = -2,    /* D != 64, or the device is not sm_100 */
     HMAR_ERR_CUDA = -3,           /* a CUDA runtime / driver call failed */
     HMAR_ERR_WORKSPACE = -4,      /* workspace missing or smaller than hmar_attn_bwd_workspace_bytes() */
-    HMAR_ERR_DEVICE_TIMEOUT = -5  /* a bounded wait inside a kernel ran out (see hmar_device_status) */
+    HMAR_ERR_DEVICE_TIMEOUT = -5, /* a bounded wait inside a kernel ran out (see hmar_device_status) */
+    HMAR_ERR_BOUNDS = -6          /* checking build only: a kernel formed an address outside its tensor (hmar_device_status) */
 } hmar_status;
 
 #define HMAR_MAX_SCALES 64

@@ -20,6 +20,7 @@ HMAR_ERR_UNSUPPORTED = -2
 HMAR_ERR_CUDA = -3
 HMAR_ERR_WORKSPACE = -4
 HMAR_ERR_DEVICE_TIMEOUT = -5
+HMAR_ERR_BOUNDS = -6
 
 HMAR_WINDOW_MARKOV = 0      # scales k-1 and k (HMAR)
 HMAR_WINDOW_CAUSAL = 1      # scales 1..k (VAR's block-causal mask)
@@ -46,8 +47,11 @@ def lib():
     global _LIB
     if _LIB is not None:
         return _LIB
-    path = _build.LIB_PATH
-    if _build.needs_build():
+    path = _build.LIB_PATH                 # libhmar.so, or the library named by the HMAR_LIBRARY environment variable
+    if os.path.abspath(path) == os.path.abspath(_build.CHECKED_LIB_PATH):
+        if _build.needs_build(path):
+            path = _build.build(checked=True)
+    elif "HMAR_LIBRARY" not in os.environ and _build.needs_build():
         path = _build.build()
     L = ctypes.CDLL(path)
     vp, ip, fp = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int), ctypes.c_float

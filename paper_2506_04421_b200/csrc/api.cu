@@ -364,7 +364,7 @@ int hmar_device_status(int* detail) {
     const int zero[2] = {0, 0};
     if (cudaMemcpyToSymbol(g_device_status, zero, sizeof(zero)) != cudaSuccess) { cudaGetLastError(); return HMAR_ERR_CUDA; }
     if (detail) *detail = host[1];
-    return host[0] == 0 ? HMAR_OK : HMAR_ERR_DEVICE_TIMEOUT;
+    return host[0];
 }
 
 void hmar_profile_begin(void) {
@@ -442,6 +442,7 @@ const char* hmar_status_string(int status) {
         case HMAR_ERR_CUDA: return "CUDA call failed";
         case HMAR_ERR_WORKSPACE: return "workspace missing or too small";
         case HMAR_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel ran out";
+        case HMAR_ERR_BOUNDS: return "checking build: a kernel formed an address outside its tensor";
         default: return "unknown status";
     }
 }

@@ -388,7 +388,8 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
 #pragma unroll
                     for (int t = 0; t < BQ / 32; ++t) {
                         const int row = q0 + t * 32 + lane;
-                        const bool in = row < w.q_end;
+                        const bool in = row < w.q_end &&
+                                        HMAR_IN_BOUNDS(row >= 0 && row < L && bh >= 0 && bh < args.n_heads, args.status, 0xB201);
                         lv[t] = in ? __ldg(args.lse + (size_t)bh * L + row) : INFINITY;
                         dv[t] = in ? __ldg(args.delta + (size_t)bh * L + row) : 0.f;
                     }
@@ -589,9 +590,11 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             } else {
                 vsrc = reinterpret_cast<const uint4*>(args.v + ((size_t)(gc / n_work) * L + row) * D);
             }
+            const long long v_off = reinterpret_cast<const __nv_bfloat16*>(vsrc) - args.v;
+            const bool v_in = row < L && HMAR_IN_BOUNDS(v_off >= 0 && v_off + D <= args.in_extent, args.status, 0xB202);
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
-                const uint4 val = row < L ? __ldg(vsrc + c) : make_uint4(0u, 0u, 0u, 0u);
+                const uint4 val = v_in ? __ldg(vsrc + c) : make_uint4(0u, 0u, 0u, 0u);
                 buf[4 * c] = val.x; buf[4 * c + 1] = val.y; buf[4 * c + 2] = val.z; buf[4 * c + 3] = val.w;
             }
             if (wait_free) {
@@ -652,8 +655,10 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                             } else {
                                 dst = reinterpret_cast<uint4*>(base + ((size_t)bh * L + w.row_begin + r) * D + (part & 1) * 32);
                             }
+                            const long long g_off = reinterpret_cast<__nv_bfloat16*>(dst) - base;
+                            const bool g_in = HMAR_IN_BOUNDS(g_off >= 0 && g_off + 32 <= args.g_extent, args.status, 0xB203);
 #pragma unroll
-                            for (int t = 0; t < 4; ++t) {
+                            for (int t = 0; t < 4 && g_in; ++t) {
                                 uint4 o;
                                 o.x = pack_bf16(__uint_as_float(buf[8 * t + 0]) * mul, __uint_as_float(buf[8 * t + 1]) * mul);
                                 o.y = pack_bf16(__uint_as_float(buf[8 * t + 2]) * mul, __uint_as_float(buf[8 * t + 3]) * mul);

@@ -418,10 +418,11 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             tmem_ld32(o_addr, b0);
             tmem_ld32(o_addr + 32, b1);
             tmem_ld_wait();
-            if (row_ok) {
-                __nv_bfloat16* orow = args.out + batch * args.out_batch_stride + head * args.out_head_stride +
-                                      row * args.out_row_stride;
-                uint4* dst = reinterpret_cast<uint4*>(orow);
+            const long long out_off = batch * args.out_batch_stride + head * args.out_head_stride + row * args.out_row_stride;
+            const long long lse_off = (long long)bh * args.n_q_rows + row;
+            if (row_ok && HMAR_IN_BOUNDS(out_off >= 0 && out_off + D <= args.out_extent, args.status, 0xB101) &&
+                HMAR_IN_BOUNDS(args.lse == nullptr || (lse_off >= 0 && lse_off < args.lse_extent), args.status, 0xB102)) {
+                uint4* dst = reinterpret_cast<uint4*>(args.out + out_off);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     uint4 v4;
@@ -441,7 +442,7 @@ hmar_fwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
                     dst[4 + i] = v4;
                 }
                 if (args.lse != nullptr)
-                    args.lse[(size_t)bh * args.n_q_rows + row] = (m_used + log2f(l)) * 0.6931471805599453f;
+                    args.lse[lse_off] = (m_used + log2f(l)) * 0.6931471805599453f;
             }
         }
     }

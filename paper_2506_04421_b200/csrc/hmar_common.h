@@ -56,6 +56,23 @@ void build_scale_table(int n_scales, const int* side_lens, int window, ScaleTabl
 std::vector<Tile> build_tiles(const ScaleTable& st, int direction);
 
 #if defined(__CUDACC__)
+// Checking build (-DHMAR_BOUNDS_CHECK, a separate library used by the tests): every address the kernels form by
+// their own arithmetic for a plain load or store (TMA copies are clipped by the hardware against the tensor map)
+// is compared with the extent of its tensor first.  An offset outside records HMAR_ERR_BOUNDS with the site's
+// code in the status word and the access is skipped; nothing traps.  In the normal build the check folds away.
+#if defined(HMAR_BOUNDS_CHECK)
+__device__ __forceinline__ bool hmar_bounds_fail(int* status, int site) {
+    if (status != nullptr) {
+        atomicCAS(status, 0, HMAR_ERR_BOUNDS);
+        atomicCAS(status + 1, 0, site);
+    }
+    return false;
+}
+#define HMAR_IN_BOUNDS(cond, status, site) ((cond) ? true : hmar_bounds_fail((status), (site)))
+#else
+#define HMAR_IN_BOUNDS(cond, status, site) true
+#endif
+
 __device__ __forceinline__ int scale_of_row(const ScaleTable& st, int row) {
     int s = 0;
     while (s + 1 < st.n_scales && row >= st.start[s + 1]) ++s;

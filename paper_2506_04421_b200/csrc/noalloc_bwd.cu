@@ -148,6 +148,7 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
     a.in_row = a.od_row = a.g_row = kHeadDim;
     a.in_head = a.od_head = a.g_head = L * kHeadDim;
     a.in_batch = a.od_batch = a.g_batch = (long long)BH * L * kHeadDim;
+    a.in_extent = a.g_extent = (long long)BH * L * kHeadDim;
     a.v = static_cast<const __nv_bfloat16*>(v);
     a.dk = static_cast<__nv_bfloat16*>(dk);
     a.dv = static_cast<__nv_bfloat16*>(dv);

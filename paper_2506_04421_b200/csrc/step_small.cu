@@ -52,6 +52,8 @@ struct StepArgs {
     long long q_head_stride, kv_prev_head_stride, kv_cur_head_stride, out_head_stride;    // elements
     int n_prev, n_cur;
     float scale_log2;
+    int n_heads;
+    int* status;                // device status word (checking build), may be nullptr
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t smem_addr, const void* gptr) {
@@ -65,6 +67,7 @@ __global__ void __launch_bounds__(kSmallMaxQueries, 4)
 hmar_step_small_kernel(const StepArgs a) {
     extern __shared__ __align__(16) uint8_t smem[];
     const int bh = blockIdx.x;
+    if (!HMAR_IN_BOUNDS(bh < a.n_heads && a.n_cur <= kSmallMaxQueries && a.n_prev + a.n_cur <= kSmallMaxKeys, a.status, 0xB301)) return;
     const int n_keys = a.n_prev + a.n_cur;
     const int keys_pad = (n_keys + 15) & ~15;
     uint8_t* sk = smem;
@@ -221,7 +224,7 @@ hmar_step_small_kernel(const StepArgs a) {
 #pragma unroll
         for (int d = 0; d < 8; ++d) {
             const int c = d * 8 + t * 2;
-            if (row0 < a.n_cur) *reinterpret_cast<uint32_t*>(oh + (size_t)row0 * D + c) = pack2(o[r][d][0] * inv0, o[r][d][1] * inv0);
+            if (row0 < a.n_cur && HMAR_IN_BOUNDS(c + 2 <= D, a.status, 0xB302)) *reinterpret_cast<uint32_t*>(oh + (size_t)row0 * D + c) = pack2(o[r][d][0] * inv0, o[r][d][1] * inv0);
             if (row1 < a.n_cur) *reinterpret_cast<uint32_t*>(oh + (size_t)row1 * D + c) = pack2(o[r][d][2] * inv1, o[r][d][3] * inv1);
         }
         if (a.lse != nullptr && t == 0) {
@@ -238,7 +241,7 @@ bool step_small_applies(int n_prev, int n_cur) { return n_prev + n_cur <= kSmall
 int step_small(const __nv_bfloat16* q, const __nv_bfloat16* k_prev, const __nv_bfloat16* v_prev,
                const __nv_bfloat16* k_cur, const __nv_bfloat16* v_cur, __nv_bfloat16* out, float* lse, int BH, int n_prev,
                int n_cur, long long q_head_stride, long long kv_prev_head_stride, long long kv_cur_head_stride,
-               long long out_head_stride, float scale, cudaStream_t stream) {
+               long long out_head_stride, float scale, int* status, cudaStream_t stream) {
     StepArgs a;
     a.q = q; a.k_prev = k_prev; a.v_prev = v_prev; a.k_cur = k_cur; a.v_cur = v_cur;
     a.out = out; a.lse = lse;
@@ -246,6 +249,8 @@ int step_small(const __nv_bfloat16* q, const __nv_bfloat16* k_prev, const __nv_b
     a.kv_cur_head_stride = kv_cur_head_stride; a.out_head_stride = out_head_stride;
     a.n_prev = n_prev; a.n_cur = n_cur;
     a.scale_log2 = scale * 1.4426950408889634f;
+    a.n_heads = BH;
+    a.status = status;
     const int warps = (n_cur + 31) / 32;
     const int keys_pad = (n_prev + n_cur + 15) & ~15;
     const size_t smem = (size_t)2 * keys_pad * ROW_BYTES;

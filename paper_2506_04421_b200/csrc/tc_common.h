@@ -23,6 +23,7 @@ struct FwdArgs {
     int n_q_rows;            // rows per head of q / out / lse
     int heads_per_batch;     // H: head bh is head bh % H of batch bh / H (the tensor maps are 4-D: D, rows, H, B)
     long long out_row_stride, out_head_stride, out_batch_stride;   // of `out`, in elements (lse is always [B*H, rows])
+    long long out_extent, lse_extent;   // elements reachable through out / lse (read by the checking build only)
     int n0, n1;              // inference step: rows of the previous / current scale's keys
     float scale_log2;        // softmax_scale * log2(e)
     __nv_bfloat16* out;
@@ -72,6 +73,7 @@ struct BwdArgs {
     long long in_row, in_head, in_batch;
     long long od_row, od_head, od_batch;
     long long g_row, g_head, g_batch;
+    long long in_extent, g_extent;      // elements reachable through v and through dk / dv (checking build only)
     const __nv_bfloat16* v;  // read directly for the rows that go to TMEM
     __nv_bfloat16* dk;
     __nv_bfloat16* dv;

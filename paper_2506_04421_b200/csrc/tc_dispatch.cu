@@ -190,6 +190,8 @@ static int tc_fwd_strided(const bf16* q, const bf16* k, const bf16* v, bf16* out
     a.out_row_stride = out_row;
     a.out_head_stride = out_head;
     a.out_batch_stride = out_batch;
+    a.out_extent = (B - 1) * out_batch + (H - 1) * out_head + (long long)(L - 1) * out_row + kHeadDim;
+    a.lse_extent = (long long)B * H * L;
     a.n0 = L;
     a.n1 = 0;
     a.scale_log2 = scale * 1.4426950408889634f;
@@ -221,7 +223,7 @@ int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const b
                   cudaStream_t stream) {
     if (step_small_applies(n_prev, n_cur))
         return step_small(q, k_prev, v_prev, k_cur, v_cur, out, lse, BH, n_prev, n_cur, st.q, st.kv_prev, st.kv_cur, st.out,
-                          scale, stream);
+                          scale, status, stream);
     CUtensorMap mq, mk0, mv0, mk1, mv1;
     auto rows_map = [&](CUtensorMap* m, const bf16* base, int rows, long long head_stride, int box_rows) {
         return make_rows_map4(m, base, 1, BH, rows, kHeadDim, head_stride, (long long)BH * head_stride, box_rows);
@@ -244,6 +246,8 @@ int tc_scale_step(const bf16* q, const bf16* k_prev, const bf16* v_prev, const b
     a.out_row_stride = kHeadDim;
     a.out_head_stride = st.out;
     a.out_batch_stride = (long long)BH * st.out;
+    a.out_extent = (long long)(BH - 1) * st.out + (long long)n_cur * kHeadDim;
+    a.lse_extent = (long long)BH * n_cur;
     a.n0 = n_prev;
     a.n1 = n_cur;
     a.scale_log2 = scale * 1.4426950408889634f;
@@ -287,6 +291,8 @@ static int tc_bwd_strided(const bf16* q, const bf16* k, const bf16* v, const bf1
     a.in_row = in.row; a.in_head = in.head; a.in_batch = in.batch;
     a.od_row = od.row; a.od_head = od.head; a.od_batch = od.batch;
     a.g_row = g.row; a.g_head = g.head; a.g_batch = g.batch;
+    a.in_extent = (B - 1) * in.batch + (H - 1) * in.head + (long long)(L - 1) * in.row + kHeadDim;
+    a.g_extent = (B - 1) * g.batch + (H - 1) * g.head + (long long)(L - 1) * g.row + kHeadDim;
     a.v = v;
     a.dk = dk;
     a.dv = dv;

@@ -35,7 +35,7 @@ bool step_small_applies(int n_prev, int n_cur);
 int step_small(const __nv_bfloat16* q, const __nv_bfloat16* k_prev, const __nv_bfloat16* v_prev,
                const __nv_bfloat16* k_cur, const __nv_bfloat16* v_cur, __nv_bfloat16* out, float* lse, int BH, int n_prev,
                int n_cur, long long q_head_stride, long long kv_prev_head_stride, long long kv_cur_head_stride,
-               long long out_head_stride, float scale, cudaStream_t stream);
+               long long out_head_stride, float scale, int* status, cudaStream_t stream);
 void tc_release_plans();
 
 }  // namespace hmar

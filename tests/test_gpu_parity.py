@@ -601,3 +601,24 @@ def test_recon_accumulate_matches_oracle(side, out_side, B, C, V, masked):
     err = np.abs(xhat.double().cpu().numpy() - ref)
     assert err.max() <= 1e-5 * max(1.0, np.abs(ref).max()), f"max abs err {err.max():.3e}"
     assert all(intact() for intact in guards)
+
+
+def test_edge_cases_through_the_checking_build():
+    """The library compiled with -DHMAR_BOUNDS_CHECK compares every address its kernels form by their own
+    arithmetic (plain loads and stores; TMA copies are clipped by the hardware) with the extent of its tensor and
+    records HMAR_ERR_BOUNDS instead of accessing.  The edge-case side lists, the packed layouts, the K/V ring and
+    the small-window step run through it in a fresh process; _no_device_error() in those tests fails on any
+    recorded code, and the results still have to match the oracle."""
+    import os
+    import subprocess
+    import sys
+    from paper_2506_04421_b200 import build as b
+    lib_path = b.build(checked=True)
+    env = dict(os.environ, HMAR_LIBRARY=lib_path)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    sel = "test_edge_side_lists_fwd_bwd or test_config1 or test_packed_qkv_backward or test_scale_step_on_a_kv_ring or " \
+          "test_scale_step_small_batch_all_scales or test_other_block_masks_fwd_bwd"
+    res = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_parity.py"), "-x", "-q", "-m", "gpu",
+                          "-k", sel, "-p", "no:cacheprovider"], env=env, capture_output=True, text=True, cwd=root, timeout=900)
+    assert res.returncode == 0, res.stdout[-3000:] + res.stderr[-1000:]
+    assert " passed" in res.stdout
