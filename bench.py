@@ -250,6 +250,41 @@ def time_small_config(hmar, wl_x, dev, peaks, reps=4):
     return res
 
 
+def time_recon(hmar, dev, peaks, reps=20):
+    """The sampler's neighbour step (Alg. 2 lines 7-8 fused with the sub-step's token selection) on a synthetic
+    codebook (V = 4096, C = 32), latent 32 x 32: at the sampler's batch (64) and at a batch whose reconstruction
+    exceeds L2 (2048: 268 MB), for the last scale (32 -> 32) and a middle one (13 -> 32).  GB/s on the algorithmic
+    bytes (the reconstruction read and written once) against the measured HBM bandwidth."""
+    import torch
+    rows = []
+    g = torch.Generator(device=dev)
+    g.manual_seed(4421)
+    V, C, S = 4096, 32, 32
+    codebook = torch.randn((V, C), generator=g, device=dev)
+    for B in (64, 2048):
+        xhat = torch.zeros((B, C, S, S), device=dev)
+        for side in (13, 32):
+            old = torch.randint(0, V, (B, side, side), generator=g, device=dev, dtype=torch.int32)
+            new = torch.randint(0, V, (B, side, side), generator=g, device=dev, dtype=torch.int32)
+            mask = torch.randint(0, 2, (B, side, side), generator=g, device=dev, dtype=torch.uint8)
+            sel = torch.empty_like(old)
+            for _ in range(3):
+                hmar.hmar_recon_accumulate(xhat, codebook, new, old, mask, sel)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                hmar.hmar_recon_accumulate(xhat, codebook, new, old, mask, sel)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / reps
+            byt = 2 * xhat.numel() * 4
+            rows.append({"B": B, "side": side, "ms": round(ms, 4), "gbs": round(byt / ms / 1e6, 1),
+                         "frac_hbm": round(byt / ms / 1e6 / peaks["hbm_gbs"], 4), "algorithmic_bytes": byt})
+        del xhat
+        torch.cuda.empty_cache()
+    return rows
+
+
 def oracle_errors(hmar, dev):
     """Max / mean abs error against the CPU oracle of one head per config, the head placed in an otherwise
     device-generated full-size problem (outside every timed region)."""
@@ -475,6 +510,7 @@ def run_ours(args, wl):
             for nm in ("256_d16_fwd", "256_d30_train"):
                 extras[nm] = time_small_config(hmar, CONFIGS[nm], dev, peaks)
                 torch.cuda.empty_cache()
+            extras["recon_accumulate"] = {"workload": "synthetic codebook V=4096 C=32, latent 32x32", "rows": time_recon(hmar, dev, peaks)}
             try:
                 extras["oracle_errors"] = oracle_errors(hmar, dev)
             except Exception as e:     # context; its failure must not lose the benchmark line

@@ -129,3 +129,38 @@ def test_valid_call_without_a_device_fails_loudly():
     if torch.cuda.is_available():
         pytest.skip("a device is present")
     assert _call_fwd() in (hmar.HMAR_ERR_CUDA, hmar.HMAR_ERR_UNSUPPORTED)
+
+
+def test_argument_errors_of_the_added_entry_points():
+    """Validation runs before any device is touched (the pointers are fake and never dereferenced)."""
+    L = hmar.lib()
+    p = ctypes.c_void_p(1 << 12)
+    sides = (ctypes.c_int * 2)(1, 2)
+    # packed backward
+    f = L.hmar_attn_bwd_packed
+    assert f(None, p, p, p, p, p, 1 << 20, 1, 1, 64, 2, sides, 0.125, None) == hmar.HMAR_ERR_BAD_ARG
+    assert f(p, p, p, p, p, p, 1 << 20, 1, 1, 128, 2, sides, 0.125, None) == hmar.HMAR_ERR_UNSUPPORTED
+    assert f(p, p, p, p, p, None, 0, 1, 1, 64, 2, sides, 0.125, None) == hmar.HMAR_ERR_WORKSPACE
+    assert f(p, p, p, p, p, p, 16, 1, 1, 64, 2, sides, 0.125, None) == hmar.HMAR_ERR_WORKSPACE
+    # the fourth window is accepted by the scheduler, a fifth is not
+    assert L.hmar_schedule_tiles_window(2, sides, hmar.HMAR_WINDOW_PREV, 1, None, 0) > 0
+    assert L.hmar_schedule_tiles_window(2, sides, 4, 1, None, 0) == hmar.HMAR_ERR_BAD_ARG
+    # reconstruction step
+    g = L.hmar_recon_accumulate
+    assert g(None, p, None, p, None, None, 1, 32, 4096, 4, 32, None) == hmar.HMAR_ERR_BAD_ARG        # no xhat
+    assert g(p, p, None, p, None, None, 1, 32, 4096, 33, 32, None) == hmar.HMAR_ERR_BAD_ARG          # would shrink the map
+    assert g(p, p, None, p, p, None, 1, 32, 4096, 4, 32, None) == hmar.HMAR_ERR_BAD_ARG              # mask without old tokens
+    assert g(p, p, p, p, p, p, 1, 32, 4096, 4, 32, None) == hmar.HMAR_ERR_BAD_ARG                    # tokens_out aliases an input
+    assert g(p, p, None, p, None, None, 0, 32, 4096, 4, 32, None) == hmar.HMAR_ERR_BAD_ARG
+
+
+def test_prev_window_backward_tiles_leave_out_nothing_but_the_last_scale():
+    # under the preceding-scale mask the only key rows without queries are those of the last scale
+    for sides in ((3, 11, 12), (1, 2, 3, 4, 6, 9, 13, 18), (12, 12, 12)):
+        tiles = hmar.hmar_schedule_tiles(sides, 1, window=hmar.HMAR_WINDOW_PREV)
+        empty = [t for t in tiles if t["partner_begin"] == t["partner_end"]]
+        L_total = sum(s * s for s in sides)
+        last_begin = L_total - sides[-1] ** 2
+        assert all(t["row_begin"] >= last_begin for t in empty)
+        covered = sum(t["row_count"] for t in empty)
+        assert covered <= sides[-1] ** 2
