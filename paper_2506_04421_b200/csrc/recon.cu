@@ -8,8 +8,10 @@
 // (a = -0.75, half-pixel sample positions, border indices clamped) and add the result to the running
 // reconstruction in place.  The reconstruction is read and written exactly once (the algorithmic HBM bytes
 // of the step); the codebook (V x C fp32, 512 KB for V = 4096, C = 32) and the token maps stay in L2 / L1.
-// A thread owns one output pixel and walks the channels, so a warp's accesses to the [B, C, H, W] tensor
-// are 128-byte rows for every channel.
+// Two kernels: for token maps of at most 32 x 32 (every scale of the paper's schedules) a block takes one image
+// and stages the looked-up coarse map in shared memory; larger maps go through the plain kernel, in which a
+// thread owns one output pixel and walks the channels.  In both a warp's accesses to the [B, C, H, W] tensor
+// are 128-byte rows.
 #include <cuda_runtime.h>
 
 #include "hmar_common.h"
@@ -72,11 +74,87 @@ hmar_recon_accumulate_kernel(float* __restrict__ xhat, const float* __restrict__
     }
 }
 
+// Staged variant for token maps of at most 32 x 32: one block per image and group of 8 channels.  The selected
+// tokens' code values are gathered once into shared memory as a channel-major coarse map (rows padded by one word,
+// so the transposing stores spread over the banks), then every warp takes (channel, output row) pairs: 16 taps
+// from shared memory per output pixel and one 128-byte read-modify-write of the reconstruction per row.  Each
+// code vector is fetched once per image instead of once per output pixel and tap, and a launch at the sampler's
+// batch still has a few hundred blocks.
+constexpr int kStageMaxSide = 32;
+constexpr int kStageChannels = 8;
+
+__global__ void __launch_bounds__(256)
+hmar_recon_accumulate_staged_kernel(float* __restrict__ xhat, const float* __restrict__ codebook,
+                                    const int* __restrict__ tokens_old, const int* __restrict__ tokens_new,
+                                    const unsigned char* __restrict__ mask, int* __restrict__ tokens_out,
+                                    int C, int V, int side, int out_side, int n_groups) {
+    __shared__ float coarse[kStageChannels * (kStageMaxSide * kStageMaxSide + 1)];
+    __shared__ int ids[kStageMaxSide * kStageMaxSide];
+    const int b = blockIdx.x / n_groups, grp = blockIdx.x - b * n_groups;
+    const int c0 = grp * kStageChannels, nc = min(kStageChannels, C - c0);
+    const int n_tok = side * side, stride = n_tok + 1;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    // ---- token selection (written out by the image's first channel group)
+    for (int pos = threadIdx.x; pos < n_tok; pos += blockDim.x) {
+        const long long gp = (long long)b * n_tok + pos;
+        const int t = (mask == nullptr || mask[gp] != 0) ? tokens_new[gp] : tokens_old[gp];
+        if (tokens_out != nullptr && grp == 0) tokens_out[gp] = t;
+        ids[pos] = min(max(t, 0), V - 1);
+    }
+    __syncthreads();
+    // ---- gather: a thread per (token, channel): 8 consecutive lanes read one token's 8 channels (32 bytes)
+    for (int idx = threadIdx.x; idx < n_tok * kStageChannels; idx += blockDim.x) {
+        const int pos = idx / kStageChannels, ch = idx - pos * kStageChannels;
+        if (ch < nc) coarse[ch * stride + pos] = __ldg(codebook + (long long)ids[pos] * C + c0 + ch);
+    }
+    __syncthreads();
+    // ---- interpolate and accumulate: lane per output column, warp per (channel, output row)
+    const float ratio = (float)side / (float)out_side;
+    const long long plane = (long long)out_side * out_side;
+    for (int ox = lane; ox < out_side; ox += 32) {
+        const float sx = (ox + 0.5f) * ratio - 0.5f;
+        const int ix = (int)floorf(sx);
+        float wx[4];
+        cubic_weights(sx - (float)ix, wx);
+        int xx[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) xx[c] = min(max(ix - 1 + c, 0), side - 1);
+        for (int task = warp; task < nc * out_side; task += n_warps) {
+            const int ch = task / out_side, oy = task - ch * out_side;
+            const float sy = (oy + 0.5f) * ratio - 0.5f;
+            const int iy = (int)floorf(sy);
+            float wy[4];
+            cubic_weights(sy - (float)iy, wy);
+            const float* src = coarse + ch * stride;
+            float acc = 0.f;
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                const float* row = src + min(max(iy - 1 + a, 0), side - 1) * side;
+                float h = 0.f;                              // the row's four taps first, then its weight
+#pragma unroll
+                for (int c = 0; c < 4; ++c) h = fmaf(wx[c], row[xx[c]], h);
+                acc = fmaf(wy[a], h, acc);
+            }
+            xhat[((long long)b * C + c0 + ch) * plane + (long long)oy * out_side + ox] += acc;
+        }
+    }
+}
+
 }  // namespace
 
 cudaError_t launch_recon_accumulate(float* xhat, const float* codebook, const int* tokens_old, const int* tokens_new,
                                     const unsigned char* mask, int* tokens_out, int B, int C, int V, int side, int out_side,
                                     cudaStream_t stream) {
+    if (side <= kStageMaxSide) {
+        const int n_groups = (C + kStageChannels - 1) / kStageChannels;
+        {
+            KernelTimer timer("hmar_recon_accumulate_kernel", stream);
+            hmar_recon_accumulate_staged_kernel<<<(unsigned)B * n_groups, 256, 0, stream>>>(xhat, codebook, tokens_old, tokens_new, mask,
+                                                                                            tokens_out, C, V, side, out_side, n_groups);
+        }
+        count_launch(1);
+        return cudaGetLastError();
+    }
     const long long n_pix = (long long)B * out_side * out_side;
     const unsigned grid = (unsigned)((n_pix + 255) / 256);
     {

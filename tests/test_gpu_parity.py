@@ -578,11 +578,12 @@ def test_repeat_calls_are_stable():
 
 
 @pytest.mark.parametrize("side,out_side,B,C,V", [(1, 32, 3, 32, 4096), (6, 32, 2, 32, 4096), (13, 32, 2, 32, 4096), (32, 32, 2, 32, 4096),
-                                                  (3, 7, 2, 5, 17), (16, 16, 65, 32, 4096)])
+                                                  (3, 7, 2, 5, 17), (16, 16, 65, 32, 4096), (5, 16, 2, 40, 33), (40, 48, 1, 8, 50)])
 @pytest.mark.parametrize("masked", [False, True])
 def test_recon_accumulate_matches_oracle(side, out_side, B, C, V, masked):
     """The sampler's neighbour step (Alg. 2 lines 7-8 with the sub-step's token selection, Sec. 4.2) on a synthetic
-    codebook: fp32 on the GPU against the fp64 oracle, and the selected token map bit for bit."""
+    codebook: fp32 on the GPU against the fp64 oracle, and the selected token map bit for bit.  Maps of at most
+    32 x 32 tokens take the staged kernel (also with more than 32 channels), the 40 x 40 case the plain one."""
     rng = np.random.default_rng(1000 * side + out_side + int(masked))
     codebook = rng.standard_normal((V, C)).astype(np.float32)
     old = rng.integers(0, V, (B, side, side)).astype(np.int32)
