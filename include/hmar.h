@@ -41,7 +41,7 @@ extern "C" {
 typedef enum {
     HMAR_OK = 0,
     HMAR_ERR_BAD_ARG = -1,        /* null pointer, non-positive size, misaligned pointer, too many scales */
-    HMAR_ERR_UNSUPPORTED = -2,    /* D != 64, or the device is not sm_100 */
+    HMAR_ERR_UNSUPPORTED = -2,    /* head dimension not offered by this entry point, or the device is not sm_100 */
     HMAR_ERR_CUDA = -3,           /* a CUDA runtime / driver call failed */
     HMAR_ERR_WORKSPACE = -4,      /* workspace missing or smaller than hmar_attn_bwd_workspace_bytes() */
     HMAR_ERR_DEVICE_TIMEOUT = -5, /* a bounded wait inside a kernel ran out (see hmar_device_status) */
@@ -62,6 +62,12 @@ typedef enum {
  *                        scale, which has no predecessor, attends to itself.  No query looks at the keys of the
  *                        last scale, so the backward returns zeros for their dK and dV. */
 typedef enum { HMAR_WINDOW_MARKOV = 0, HMAR_WINDOW_CAUSAL = 1, HMAR_WINDOW_SELF = 2, HMAR_WINDOW_PREV = 3 } hmar_window;
+
+/* Head dimension D.  The tensor-core kernels exist for D = 64 (the paper's attention benchmark, App. B.4, and
+ * every config).  hmar_attn_fwd, hmar_attn_bwd, their _window and _f32 forms, hmar_attn_bwd_workspace_bytes and
+ * hmar_attn_scale_step(_f32) also accept D = 32 and D = 128, which run on the plain-FMA kernels of the debug
+ * build (same results within the same tolerances, a small fraction of the speed).  The packed, strided and
+ * no-allocation entry points take D = 64 only.  Anything else is HMAR_ERR_UNSUPPORTED. */
 
 /* Training forward (Sec. 4.1; App. B.4 benchmarks this pass).
  *   q, k, v : [B,H,L,D] in;  out : [B,H,L,D] out;  lse : [B,H,L] fp32 out.

@@ -59,10 +59,12 @@ static int check_scale(float softmax_scale) {
     return (softmax_scale > 0.f && softmax_scale < 1e30f) ? HMAR_OK : HMAR_ERR_BAD_ARG;
 }
 
-static int check_shape(int B, int H, int D) {
+// any_d: the entry point also runs the plain kernels, which exist for head dimensions 32, 64 and 128; the
+// tensor-core kernels (and every entry point that has nothing else) take 64 only
+static int check_shape(int B, int H, int D, bool any_d = false) {
     if (B <= 0 || H <= 0 || D <= 0) return HMAR_ERR_BAD_ARG;
     if ((long long)B * H > 65535) return HMAR_ERR_BAD_ARG;   // heads map to gridDim.y
-    if (D != kHeadDim) return HMAR_ERR_UNSUPPORTED;
+    if (D != kHeadDim && !(any_d && (D == 32 || D == 128))) return HMAR_ERR_UNSUPPORTED;
     return HMAR_OK;
 }
 
@@ -111,7 +113,8 @@ static int* device_status_ptr() {
 template <typename T>
 static int fwd_impl(const T* q, const T* k, const T* v, T* out, float* lse, int B, int H, int D,
                     int n_scales, const int* side_lens, int window, float softmax_scale, void* stream, bool tensor_core) {
-    int rc = check_shape(B, H, D);
+    int rc = check_shape(B, H, D, true);
+    tensor_core = tensor_core && D == kHeadDim;
     if (rc != HMAR_OK) return rc;
     ScaleTable st;
     rc = check_sides(n_scales, side_lens, window, &st);
@@ -127,14 +130,15 @@ static int fwd_impl(const T* q, const T* k, const T* v, T* out, float* lse, int 
         if (tensor_core && !g_force_simt.load())
             return tc_fwd(q, k, v, out, lse, B * H, st, softmax_scale, device_status_ptr(), s);
     }
-    return simt_fwd<T>(q, k, v, out, lse, B * H, st, softmax_scale, s) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
+    return simt_fwd<T>(q, k, v, out, lse, B * H, D, st, softmax_scale, s) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
 template <typename T>
 static int bwd_impl(const T* q, const T* k, const T* v, const T* out, const float* lse, const T* dout,
                     T* dq, T* dk, T* dv, void* workspace, size_t workspace_bytes, int B, int H, int D,
                     int n_scales, const int* side_lens, int window, float softmax_scale, void* stream, bool tensor_core) {
-    int rc = check_shape(B, H, D);
+    int rc = check_shape(B, H, D, true);
+    tensor_core = tensor_core && D == kHeadDim;
     if (rc != HMAR_OK) return rc;
     ScaleTable st;
     rc = check_sides(n_scales, side_lens, window, &st);
@@ -159,7 +163,7 @@ static int bwd_impl(const T* q, const T* k, const T* v, const T* out, const floa
                           device_status_ptr(), s);
     }
     (void)dq_acc;
-    return simt_bwd<T>(q, k, v, out, lse, dout, dq, dk, dv, delta, B * H, st, softmax_scale, s) == cudaSuccess
+    return simt_bwd<T>(q, k, v, out, lse, dout, dq, dk, dv, delta, B * H, D, st, softmax_scale, s) == cudaSuccess
                ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
@@ -168,7 +172,8 @@ template <typename T>
 static int step_impl(const T* q, const T* k_prev, const T* v_prev, const T* k_cur, const T* v_cur, T* out,
                      float* lse, int B, int H, int D, int side_prev, int side_cur, const StepStrides* strides,
                      float softmax_scale, void* stream, bool tensor_core) {
-    int rc = check_shape(B, H, D);
+    int rc = check_shape(B, H, D, strides == nullptr);
+    tensor_core = tensor_core && D == kHeadDim;
     if (rc != HMAR_OK) return rc;
     if (side_cur <= 0 || side_cur > 4096 || side_prev < 0 || side_prev > 4096) return HMAR_ERR_BAD_ARG;
     if (check_scale(softmax_scale) != HMAR_OK) return HMAR_ERR_BAD_ARG;
@@ -200,7 +205,7 @@ static int step_impl(const T* q, const T* k_prev, const T* v_prev, const T* k_cu
                                  device_status_ptr(), s);
     }
     if (!dense) return HMAR_ERR_UNSUPPORTED;      // the plain kernels take dense tensors only
-    return simt_scale_step<T>(q, k_prev, v_prev, k_cur, v_cur, out, lse, B * H, n_prev, n_cur, softmax_scale, s)
+    return simt_scale_step<T>(q, k_prev, v_prev, k_cur, v_cur, out, lse, B * H, D, n_prev, n_cur, softmax_scale, s)
                    == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
@@ -276,9 +281,9 @@ int hmar_attn_fwd_f32(const float* q, const float* k, const float* v, float* out
 
 size_t hmar_attn_bwd_workspace_bytes(int B, int H, int D, int n_scales, const int* side_lens) {
     ScaleTable st;
-    if (check_shape(B, H, D) != HMAR_OK || check_sides(n_scales, side_lens, HMAR_WINDOW_MARKOV, &st) != HMAR_OK) return 0;
+    if (check_shape(B, H, D, true) != HMAR_OK || check_sides(n_scales, side_lens, HMAR_WINDOW_MARKOV, &st) != HMAR_OK) return 0;
     const size_t rows = (size_t)B * H * st.start[st.n_scales];
-    return round256(rows * sizeof(float)) + round256(rows * kHeadDim * sizeof(float));
+    return round256(rows * sizeof(float)) + round256(rows * D * sizeof(float));
 }
 
 int hmar_attn_bwd_window(const void* q, const void* k, const void* v, const void* out, const float* lse,

@@ -20,15 +20,15 @@ struct KernelTimer {
 };
 
 template <typename T>
-cudaError_t simt_fwd(const T* q, const T* k, const T* v, T* out, float* lse, int BH,
+cudaError_t simt_fwd(const T* q, const T* k, const T* v, T* out, float* lse, int BH, int D,
                      const ScaleTable& st, float scale, cudaStream_t stream);
 template <typename T>
 cudaError_t simt_scale_step(const T* q, const T* k_prev, const T* v_prev, const T* k_cur, const T* v_cur,
-                            T* out, float* lse, int BH, int n_prev, int n_cur, float scale,
+                            T* out, float* lse, int BH, int D, int n_prev, int n_cur, float scale,
                             cudaStream_t stream);
 template <typename T>
 cudaError_t simt_bwd(const T* q, const T* k, const T* v, const T* out, const float* lse, const T* dout,
-                     T* dq, T* dk, T* dv, float* delta, int BH, const ScaleTable& st, float scale,
+                     T* dq, T* dk, T* dv, float* delta, int BH, int D, const ScaleTable& st, float scale,
                      cudaStream_t stream);
 
 cudaError_t launch_recon_accumulate(float* xhat, const float* codebook, const int* tokens_old, const int* tokens_new,

@@ -1,6 +1,7 @@
 // Plain SIMT kernels for HMAR's Markovian masked attention: the fp32 debug build, and the bf16
 // fall-back used while debugging the tensor-core kernels.  All arithmetic is fp32 FMA; inputs and
-// outputs are float or bf16.  Two threads share one row, each owning 32 of the 64 head dimensions.
+// outputs are float or bf16.  Two threads share one row, each owning half of the head dimensions.  These
+// kernels are templated on the head dimension (32, 64, 128); the tensor-core kernels exist for 64 only.
 //
 // Mask (paper Sec. 4.1, Fig. attn-mask): a query of scale k sees keys [start[k-1], start[k+1]).
 #include <cuda_bf16.h>
@@ -11,8 +12,6 @@
 namespace hmar {
 namespace {
 
-constexpr int D = kHeadDim;
-constexpr int DH = D / 2;          // dimensions per thread
 constexpr int ROWS = 64;           // rows per block (128 threads)
 constexpr int KT = 32;             // partner rows staged in shared memory per step
 
@@ -23,7 +22,7 @@ __device__ __forceinline__ void from_f(__nv_bfloat16* p, float x) { *p = __float
 
 // Key/value rows of one head may come in two segments (previous scale, then current scale) for the
 // inference step; the training kernels use a single segment.
-template <typename T>
+template <typename T, int D>
 struct KvView {
     const T* k0; const T* v0; int n0;
     const T* k1; const T* v1;
@@ -35,7 +34,7 @@ struct KvView {
     }
 };
 
-template <typename T>
+template <typename T, int D>
 __device__ __forceinline__ void stage_rows(float (*dst)[D], const T* src_base, int first, int count) {
     // dst[r][:] = row (first + r) for r < count; 128 threads, coalesced along D
     for (int idx = threadIdx.x; idx < count * D; idx += blockDim.x) {
@@ -46,12 +45,13 @@ __device__ __forceinline__ void stage_rows(float (*dst)[D], const T* src_base, i
 
 // ---------------------------------------------------------------------------------------------
 // Forward and inference step.  dense != 0: every query row sees all n_kv keys (inference step).
-template <typename T>
+template <typename T, int D>
 __global__ void __launch_bounds__(128)
 simt_fwd_kernel(const T* __restrict__ q, const T* __restrict__ k0, const T* __restrict__ v0,
                 const T* __restrict__ k1, const T* __restrict__ v1,
                 T* __restrict__ out, float* __restrict__ lse,
                 ScaleTable st, int n_q, int n0, int n1, int dense, float scale) {
+    constexpr int DH = D / 2;          // dimensions per thread
     __shared__ float sK[KT][D];
     __shared__ float sV[KT][D];
     const int bh = blockIdx.y;
@@ -62,7 +62,7 @@ simt_fwd_kernel(const T* __restrict__ q, const T* __restrict__ k0, const T* __re
     const int row = row_ok ? row_raw : n_q - 1;
     const int last_row = min(row0 + ROWS, n_q) - 1;
 
-    KvView<T> kv{k0 + (size_t)bh * n0 * D, v0 + (size_t)bh * n0 * D, n0,
+    KvView<T, D> kv{k0 + (size_t)bh * n0 * D, v0 + (size_t)bh * n0 * D, n0,
                  k1 ? k1 + (size_t)bh * n1 * D : nullptr, v1 ? v1 + (size_t)bh * n1 * D : nullptr};
 
     int lo, hi, blk_lo, blk_hi;
@@ -122,10 +122,11 @@ simt_fwd_kernel(const T* __restrict__ q, const T* __restrict__ k0, const T* __re
 
 // ---------------------------------------------------------------------------------------------
 // delta_i = sum_d dO_id * O_id
-template <typename T>
+template <typename T, int D>
 __global__ void __launch_bounds__(128)
 simt_delta_kernel(const T* __restrict__ out, const T* __restrict__ dout, float* __restrict__ delta,
                   size_t n_rows) {
+    constexpr int DH = D / 2;          // dimensions per thread
     const size_t row = (size_t)blockIdx.x * ROWS + (threadIdx.x >> 1);
     const int half = threadIdx.x & 1;
     float acc = 0.f;
@@ -141,12 +142,13 @@ simt_delta_kernel(const T* __restrict__ out, const T* __restrict__ dout, float* 
 
 // ---------------------------------------------------------------------------------------------
 // dQ: one thread pair per query row, loop over the row's keys.
-template <typename T>
+template <typename T, int D>
 __global__ void __launch_bounds__(128)
 simt_dq_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                const T* __restrict__ dout, const float* __restrict__ lse,
                const float* __restrict__ delta, T* __restrict__ dq,
                ScaleTable st, int L, float scale) {
+    constexpr int DH = D / 2;          // dimensions per thread
     __shared__ float sK[KT][D];
     __shared__ float sV[KT][D];
     const int bh = blockIdx.y;
@@ -204,12 +206,13 @@ simt_dq_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __rest
 
 // ---------------------------------------------------------------------------------------------
 // dK, dV: one thread pair per key row, loop over the queries that see it.
-template <typename T>
+template <typename T, int D>
 __global__ void __launch_bounds__(128)
 simt_dkdv_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                  const T* __restrict__ dout, const float* __restrict__ lse,
                  const float* __restrict__ delta, T* __restrict__ dk, T* __restrict__ dv,
                  ScaleTable st, int L, float scale) {
+    constexpr int DH = D / 2;          // dimensions per thread
     __shared__ float sQ[KT][D];
     __shared__ float sG[KT][D];
     __shared__ float sLse[KT];
@@ -285,53 +288,81 @@ simt_dkdv_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __re
 // ---------------------------------------------------------------------------------------------
 // Launchers
 
-template <typename T>
-cudaError_t simt_fwd(const T* q, const T* k, const T* v, T* out, float* lse, int BH,
-                     const ScaleTable& st, float scale, cudaStream_t stream) {
+template <typename T, int D>
+static cudaError_t simt_fwd_d(const T* q, const T* k, const T* v, T* out, float* lse, int BH,
+                              const ScaleTable& st, float scale, cudaStream_t stream) {
     const int L = st.start[st.n_scales];
     dim3 grid((L + ROWS - 1) / ROWS, BH);
-    simt_fwd_kernel<T><<<grid, 128, 0, stream>>>(q, k, v, nullptr, nullptr, out, lse, st, L, L, 0, 0, scale);
+    simt_fwd_kernel<T, D><<<grid, 128, 0, stream>>>(q, k, v, nullptr, nullptr, out, lse, st, L, L, 0, 0, scale);
     count_launch(1);
     return cudaGetLastError();
 }
 
-template <typename T>
-cudaError_t simt_scale_step(const T* q, const T* k_prev, const T* v_prev, const T* k_cur, const T* v_cur,
-                            T* out, float* lse, int BH, int n_prev, int n_cur, float scale,
-                            cudaStream_t stream) {
+template <typename T, int D>
+static cudaError_t simt_scale_step_d(const T* q, const T* k_prev, const T* v_prev, const T* k_cur, const T* v_cur,
+                                     T* out, float* lse, int BH, int n_prev, int n_cur, float scale,
+                                     cudaStream_t stream) {
     ScaleTable st{};
     dim3 grid((n_cur + ROWS - 1) / ROWS, BH);
     if (n_prev > 0)
-        simt_fwd_kernel<T><<<grid, 128, 0, stream>>>(q, k_prev, v_prev, k_cur, v_cur, out, lse, st,
+        simt_fwd_kernel<T, D><<<grid, 128, 0, stream>>>(q, k_prev, v_prev, k_cur, v_cur, out, lse, st,
                                                      n_cur, n_prev, n_cur, 1, scale);
     else
-        simt_fwd_kernel<T><<<grid, 128, 0, stream>>>(q, k_cur, v_cur, nullptr, nullptr, out, lse, st,
+        simt_fwd_kernel<T, D><<<grid, 128, 0, stream>>>(q, k_cur, v_cur, nullptr, nullptr, out, lse, st,
                                                      n_cur, n_cur, 0, 1, scale);
     count_launch(1);
     return cudaGetLastError();
 }
 
-template <typename T>
-cudaError_t simt_bwd(const T* q, const T* k, const T* v, const T* out, const float* lse, const T* dout,
-                     T* dq, T* dk, T* dv, float* delta, int BH, const ScaleTable& st, float scale,
-                     cudaStream_t stream) {
+template <typename T, int D>
+static cudaError_t simt_bwd_d(const T* q, const T* k, const T* v, const T* out, const float* lse, const T* dout,
+                              T* dq, T* dk, T* dv, float* delta, int BH, const ScaleTable& st, float scale,
+                              cudaStream_t stream) {
     const int L = st.start[st.n_scales];
     const size_t n_rows = (size_t)BH * L;
-    simt_delta_kernel<T><<<(unsigned)((n_rows + ROWS - 1) / ROWS), 128, 0, stream>>>(out, dout, delta, n_rows);
+    simt_delta_kernel<T, D><<<(unsigned)((n_rows + ROWS - 1) / ROWS), 128, 0, stream>>>(out, dout, delta, n_rows);
     dim3 grid((L + ROWS - 1) / ROWS, BH);
-    simt_dq_kernel<T><<<grid, 128, 0, stream>>>(q, k, v, dout, lse, delta, dq, st, L, scale);
-    simt_dkdv_kernel<T><<<grid, 128, 0, stream>>>(q, k, v, dout, lse, delta, dk, dv, st, L, scale);
+    simt_dq_kernel<T, D><<<grid, 128, 0, stream>>>(q, k, v, dout, lse, delta, dq, st, L, scale);
+    simt_dkdv_kernel<T, D><<<grid, 128, 0, stream>>>(q, k, v, dout, lse, delta, dk, dv, st, L, scale);
     count_launch(3);
     return cudaGetLastError();
 }
 
-#define INSTANTIATE(T)                                                                                   \
-    template cudaError_t simt_fwd<T>(const T*, const T*, const T*, T*, float*, int, const ScaleTable&,   \
-                                     float, cudaStream_t);                                               \
-    template cudaError_t simt_scale_step<T>(const T*, const T*, const T*, const T*, const T*, T*, float*, \
-                                            int, int, int, float, cudaStream_t);                         \
-    template cudaError_t simt_bwd<T>(const T*, const T*, const T*, const T*, const float*, const T*, T*, \
-                                     T*, T*, float*, int, const ScaleTable&, float, cudaStream_t);
+// The public launchers pick the instantiation for the head dimension (32, 64 or 128; checked by the caller).
+#define HMAR_BY_D(call32, call64, call128) (D == 32 ? (call32) : (D == 128 ? (call128) : (call64)))
+
+template <typename T>
+cudaError_t simt_fwd(const T* q, const T* k, const T* v, T* out, float* lse, int BH, int D,
+                     const ScaleTable& st, float scale, cudaStream_t stream) {
+    return HMAR_BY_D((simt_fwd_d<T, 32>(q, k, v, out, lse, BH, st, scale, stream)), (simt_fwd_d<T, 64>(q, k, v, out, lse, BH, st, scale, stream)),
+                     (simt_fwd_d<T, 128>(q, k, v, out, lse, BH, st, scale, stream)));
+}
+
+template <typename T>
+cudaError_t simt_scale_step(const T* q, const T* k_prev, const T* v_prev, const T* k_cur, const T* v_cur,
+                            T* out, float* lse, int BH, int D, int n_prev, int n_cur, float scale,
+                            cudaStream_t stream) {
+    return HMAR_BY_D((simt_scale_step_d<T, 32>(q, k_prev, v_prev, k_cur, v_cur, out, lse, BH, n_prev, n_cur, scale, stream)),
+                     (simt_scale_step_d<T, 64>(q, k_prev, v_prev, k_cur, v_cur, out, lse, BH, n_prev, n_cur, scale, stream)),
+                     (simt_scale_step_d<T, 128>(q, k_prev, v_prev, k_cur, v_cur, out, lse, BH, n_prev, n_cur, scale, stream)));
+}
+
+template <typename T>
+cudaError_t simt_bwd(const T* q, const T* k, const T* v, const T* out, const float* lse, const T* dout,
+                     T* dq, T* dk, T* dv, float* delta, int BH, int D, const ScaleTable& st, float scale,
+                     cudaStream_t stream) {
+    return HMAR_BY_D((simt_bwd_d<T, 32>(q, k, v, out, lse, dout, dq, dk, dv, delta, BH, st, scale, stream)),
+                     (simt_bwd_d<T, 64>(q, k, v, out, lse, dout, dq, dk, dv, delta, BH, st, scale, stream)),
+                     (simt_bwd_d<T, 128>(q, k, v, out, lse, dout, dq, dk, dv, delta, BH, st, scale, stream)));
+}
+
+#define INSTANTIATE(T)                                                                                        \
+    template cudaError_t simt_fwd<T>(const T*, const T*, const T*, T*, float*, int, int, const ScaleTable&,   \
+                                     float, cudaStream_t);                                                    \
+    template cudaError_t simt_scale_step<T>(const T*, const T*, const T*, const T*, const T*, T*, float*,     \
+                                            int, int, int, int, float, cudaStream_t);                         \
+    template cudaError_t simt_bwd<T>(const T*, const T*, const T*, const T*, const float*, const T*, T*,      \
+                                     T*, T*, float*, int, int, const ScaleTable&, float, cudaStream_t);
 INSTANTIATE(float)
 INSTANTIATE(__nv_bfloat16)
 

@@ -92,8 +92,8 @@ def _no_device_error():
 
 class _Wl:
     """Ad-hoc workload for the edge-case side lists."""
-    def __init__(self, sides, B=1, H=2, seed=777):
-        self.B, self.H, self.D, self.side_lens, self.softmax_scale = B, H, 64, tuple(sides), 0.125
+    def __init__(self, sides, B=1, H=2, seed=777, D=64):
+        self.B, self.H, self.D, self.side_lens, self.softmax_scale = B, H, D, tuple(sides), 0.125
         self.seed = seed + sum((i + 1) * s for i, s in enumerate(sides))
         self.L = sum(s * s for s in sides)
 
@@ -148,6 +148,26 @@ def test_edge_side_lists_fwd_bwd(sides, dtype):
 @pytest.mark.parametrize("sides", [(1, 2, 3, 4), (3, 11), (1, 2, 3, 4, 5, 6, 8, 10, 13, 16)])
 def test_bf16_simt_fallback_kernels(sides):
     _run_training(_Wl(sides), torch.bfloat16, simt=True)
+
+
+@pytest.mark.parametrize("D", [32, 128])
+@pytest.mark.parametrize("sides", [(1, 2, 3, 4), (3, 11), (2, 1, 3, 1, 2), (1, 2, 3, 4, 5, 6, 8, 10, 13, 16)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_other_head_dimensions_through_the_plain_kernels(sides, dtype, D):
+    """Head dimensions 32 and 128 (the tensor-core kernels are D = 64 only): forward, backward and the inference
+    step on the plain-FMA kernels, same tolerances."""
+    wl = _Wl(sides, D=D)
+    wl.softmax_scale = D ** -0.5
+    _run_training(wl, dtype)
+    is_f32 = dtype == torch.float32
+    s = len(sides) - 1
+    q, kp, vp, kc, vc = scale_step_inputs(wl, s, 0, bf16=not is_f32)
+    dev = [to_device(x, wl.B, wl.H, dtype) for x in (q, kp, vp, kc, vc)]
+    out, lse = hmar.hmar_attn_scale_step(*dev, sides[s - 1], sides[s], wl.softmax_scale)
+    ref_out, ref_lse = orc.scale_step(q, kp, vp, kc, vc, wl.softmax_scale)
+    _assert_close("step out", out, ref_out, is_f32)
+    _assert_lse(lse, ref_lse, is_f32)
+    _no_device_error()
 
 
 def test_large_logits_exercise_running_max():

@@ -88,7 +88,7 @@ def test_argument_errors_are_reported_before_any_launch():
     assert _call_fwd(q=0) == hmar.HMAR_ERR_BAD_ARG
     assert _call_fwd(q=(1 << 12) + 4) == hmar.HMAR_ERR_BAD_ARG          # misaligned
     assert _call_fwd(B=0) == hmar.HMAR_ERR_BAD_ARG
-    assert _call_fwd(D=128) == hmar.HMAR_ERR_UNSUPPORTED
+    assert _call_fwd(D=48) == hmar.HMAR_ERR_UNSUPPORTED                # head dimensions are 32, 64 or 128
     assert _call_fwd(sides=()) == hmar.HMAR_ERR_BAD_ARG
     assert _call_fwd(sides=(1, 0, 2)) == hmar.HMAR_ERR_BAD_ARG
     assert _call_fwd(sides=(1, -3)) == hmar.HMAR_ERR_BAD_ARG
@@ -98,7 +98,7 @@ def test_argument_errors_are_reported_before_any_launch():
     assert _call_fwd(scale=-0.125) == hmar.HMAR_ERR_BAD_ARG
     assert _call_fwd(scale=float("inf")) == hmar.HMAR_ERR_BAD_ARG
     assert _call_fwd(scale=float("nan")) == hmar.HMAR_ERR_BAD_ARG
-    assert hmar.hmar_attn_bwd_workspace_bytes(1, 1, 32, (1, 2)) == 0
+    assert hmar.hmar_attn_bwd_workspace_bytes(1, 1, 48, (1, 2)) == 0
     assert hmar.hmar_attn_bwd_workspace_bytes(2, 3, 64, (1, 2)) >= 2 * 3 * 5 * (64 + 1) * 4
     with pytest.raises(hmar.HmarError):
         hmar.hmar_schedule_tiles((1, 0), 0)
