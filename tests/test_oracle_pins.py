@@ -582,3 +582,52 @@ def test_select_tokens_and_recon_accumulate():
     t2 = rng.integers(0, V, (B, 5, 5))
     both = orc.recon_accumulate(orc.recon_accumulate(np.zeros((B, C, S, S)), codebook, sel, S), codebook, t2, S)
     np.testing.assert_allclose(both, orc.recon_accumulate(np.zeros((B, C, S, S)), codebook, t2, S) + (x1 - x0), rtol=1e-12, atol=1e-13)
+
+
+def test_pins_detect_planted_mistakes_in_the_added_functions(monkeypatch):
+    """The same exercise for the preceding-scale mask and the reconstruction step."""
+    def fails(test, *a):
+        try:
+            test(*a)
+        except AssertionError:
+            return True
+        return False
+
+    # (1) preceding-scale mask whose first scale sees nothing / which also sees the own scale
+    good_prev = orc.previous_scale_mask
+    monkeypatch.setattr(orc, "previous_scale_mask", lambda s: good_prev(s) & ~orc.block_diagonal_mask(s))
+    assert fails(test_window_masks_single_scale_all_dense_and_nesting) and fails(test_window_masks_pair_counts_closed_forms)
+    monkeypatch.setattr(orc, "previous_scale_mask", lambda s: orc.hmar_mask(s))
+    assert fails(test_prev_window_literals_and_locality) and fails(test_window_masks_pair_counts_closed_forms)
+    monkeypatch.setattr(orc, "previous_scale_mask", good_prev)
+
+    # (2) another cubic kernel parameter; taps in reverse order
+    good_w = orc._cubic_weights
+    monkeypatch.setattr(orc, "_cubic_weights", lambda t: good_w(t, a=-0.5))
+    assert fails(test_cubic_weights_literals_and_partition_of_unity) and fails(test_bicubic_upsample_against_the_library_routine_and_special_cases)
+    monkeypatch.setattr(orc, "_cubic_weights", lambda t: good_w(t)[::-1])
+    assert fails(test_cubic_weights_literals_and_partition_of_unity) and fails(test_bicubic_upsample_against_the_library_routine_and_special_cases)
+    monkeypatch.setattr(orc, "_cubic_weights", good_w)
+
+    # (3) sample positions without the half-pixel shift (corner-aligned instead)
+    good_up = orc.bicubic_upsample
+
+    def corner_aligned(x, out_side):
+        x = np.asarray(x, dtype=np.float64)
+        h = x.shape[-1]
+        if h == out_side or h == 1:
+            return good_up(x, out_side)
+        big = good_up(x, out_side)
+        return np.roll(big, 1, axis=-1)          # any systematic shift of the sampling grid
+    monkeypatch.setattr(orc, "bicubic_upsample", corner_aligned)
+    assert fails(test_bicubic_upsample_against_the_library_routine_and_special_cases) and fails(test_select_tokens_and_recon_accumulate)
+    monkeypatch.setattr(orc, "bicubic_upsample", good_up)
+
+    # (4) the selection inverted; the accumulation replaced by an overwrite
+    good_sel = orc.select_tokens
+    monkeypatch.setattr(orc, "select_tokens", lambda o, n, m: good_sel(n, o, m))
+    assert fails(test_select_tokens_and_recon_accumulate)
+    monkeypatch.setattr(orc, "select_tokens", good_sel)
+    good_acc = orc.recon_accumulate
+    monkeypatch.setattr(orc, "recon_accumulate", lambda x, cb, t, s: good_acc(np.zeros_like(np.asarray(x, dtype=np.float64)), cb, t, s))
+    assert fails(test_select_tokens_and_recon_accumulate)
