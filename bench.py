@@ -32,7 +32,7 @@ UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (None until a capture exists for the current kernel).
 # The captures are of the batch-4 case (traffic grows in proportion to the heads), scaled by 4 to the full batch.
-NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (234577408 + 116890624), "hmar_fwd": 4 * (82925056 + 9005056)}
+NCU_TRAFFIC_BYTES = {"hmar_bwd": 4 * (230900224 + 111457792), "hmar_fwd": 4 * (82932224 + 9546496)}
 
 
 def pairs_per_head(side_lens):
