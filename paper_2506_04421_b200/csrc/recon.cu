@@ -74,26 +74,40 @@ hmar_recon_accumulate_kernel(float* __restrict__ xhat, const float* __restrict__
     }
 }
 
-// Staged variant for token maps of at most 32 x 32: one block per image and group of 8 channels.  The selected
-// tokens' code values are gathered once into shared memory as a channel-major coarse map (rows padded by one word,
-// so the transposing stores spread over the banks), then every warp takes (channel, output row) pairs: 16 taps
-// from shared memory per output pixel and one 128-byte read-modify-write of the reconstruction per row.  Each
-// code vector is fetched once per image instead of once per output pixel and tap, and a launch at the sampler's
-// batch still has a few hundred blocks.
+// Staged variant for token maps of at most 32 x 32 and reconstructions of at most 64 x 64: one block per image
+// and group of 8 channels.  The selected tokens' code values are gathered once into shared memory as a
+// channel-major coarse map (channel rows padded to 4 words past a multiple of 32, so the transposing stores spread
+// over the banks), then every warp takes a channel and walks down the output rows, interpolating separably from
+// shared memory and adding one 128-byte row segment into the reconstruction at a time.  Each code vector is
+// fetched once per image instead of once per output pixel and tap, and a launch at the sampler's batch still has
+// a few hundred blocks.
 constexpr int kStageMaxSide = 32;
 constexpr int kStageChannels = 8;
+constexpr int kStageMaxOut = 64;
 
 __global__ void __launch_bounds__(256)
 hmar_recon_accumulate_staged_kernel(float* __restrict__ xhat, const float* __restrict__ codebook,
                                     const int* __restrict__ tokens_old, const int* __restrict__ tokens_new,
                                     const unsigned char* __restrict__ mask, int* __restrict__ tokens_out,
                                     int C, int V, int side, int out_side, int n_groups) {
-    __shared__ float coarse[kStageChannels * (kStageMaxSide * kStageMaxSide + 1)];
+    __shared__ float coarse[kStageChannels * (kStageMaxSide * kStageMaxSide + 4)];
     __shared__ int ids[kStageMaxSide * kStageMaxSide];
+    __shared__ float4 row_w[kStageMaxOut];                  // per output row: the four vertical weights ...
+    __shared__ int row_src[kStageMaxOut];                   // ... and the source row of the second one
     const int b = blockIdx.x / n_groups, grp = blockIdx.x - b * n_groups;
     const int c0 = grp * kStageChannels, nc = min(kStageChannels, C - c0);
-    const int n_tok = side * side, stride = n_tok + 1;
+    const int n_tok = side * side;
+    const int stride = n_tok + ((4 - n_tok) & 31);          // = 4 mod 32: the gather's transposing stores miss each other's banks
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, n_warps = blockDim.x >> 5;
+    const float ratio = (float)side / (float)out_side;
+    if (threadIdx.x < out_side) {
+        const float sy = (threadIdx.x + 0.5f) * ratio - 0.5f;
+        const int iy = (int)floorf(sy);
+        float wy[4];
+        cubic_weights(sy - (float)iy, wy);
+        row_w[threadIdx.x] = make_float4(wy[0], wy[1], wy[2], wy[3]);
+        row_src[threadIdx.x] = iy;
+    }
     // ---- token selection (written out by the image's first channel group)
     for (int pos = threadIdx.x; pos < n_tok; pos += blockDim.x) {
         const long long gp = (long long)b * n_tok + pos;
@@ -102,14 +116,31 @@ hmar_recon_accumulate_staged_kernel(float* __restrict__ xhat, const float* __res
         ids[pos] = min(max(t, 0), V - 1);
     }
     __syncthreads();
-    // ---- gather: a thread per (token, channel): 8 consecutive lanes read one token's 8 channels (32 bytes)
-    for (int idx = threadIdx.x; idx < n_tok * kStageChannels; idx += blockDim.x) {
-        const int pos = idx / kStageChannels, ch = idx - pos * kStageChannels;
-        if (ch < nc) coarse[ch * stride + pos] = __ldg(codebook + (long long)ids[pos] * C + c0 + ch);
+    // ---- gather: a pair of lanes per token reads the group's 8 channels (32 bytes, one sector) as two 16-byte
+    // loads, so that one instruction of a warp covers 16 whole sectors; a group cut short by C, or a codebook
+    // whose rows do not start on 16-byte boundaries, goes one value at a time
+    if (nc == kStageChannels && (C & 3) == 0 && (reinterpret_cast<unsigned long long>(codebook) & 15ull) == 0) {
+#pragma unroll 4
+        for (int idx = threadIdx.x; idx < 2 * n_tok; idx += blockDim.x) {
+            const int pos = idx >> 1, half = idx & 1;
+            const float4 v = __ldg(reinterpret_cast<const float4*>(codebook + (long long)ids[pos] * C + c0) + half);
+            float* dst = coarse + (half * 4) * stride + pos;
+            dst[0 * stride] = v.x; dst[1 * stride] = v.y; dst[2 * stride] = v.z; dst[3 * stride] = v.w;
+        }
+    } else {
+        for (int idx = threadIdx.x; idx < n_tok * kStageChannels; idx += blockDim.x) {
+            const int pos = idx / kStageChannels, ch = idx - pos * kStageChannels;
+            if (ch < nc) coarse[ch * stride + pos] = __ldg(codebook + (long long)ids[pos] * C + c0 + ch);
+        }
     }
     __syncthreads();
-    // ---- interpolate and accumulate: lane per output column, warp per (channel, output row)
-    const float ratio = (float)side / (float)out_side;
+    // ---- interpolate and accumulate: lane per output column, warp per channel, walking down the output rows.
+    // The interpolation is separable: a source row's four horizontal taps are combined once (h) and reused by
+    // every output row whose vertical window holds that source row; going down, the window of four h values
+    // moves by at most one source row per output row (the step only ever enlarges a map), so an output value costs
+    // one to four shared-memory loads instead of sixteen.  Each element of the reconstruction gets exactly one
+    // addition, issued as a reduction to memory: nothing waits for the old value, and with a single addend per
+    // element the result does not depend on the order in which the reductions land.
     const long long plane = (long long)out_side * out_side;
     for (int ox = lane; ox < out_side; ox += 32) {
         const float sx = (ox + 0.5f) * ratio - 0.5f;
@@ -119,23 +150,30 @@ hmar_recon_accumulate_staged_kernel(float* __restrict__ xhat, const float* __res
         int xx[4];
 #pragma unroll
         for (int c = 0; c < 4; ++c) xx[c] = min(max(ix - 1 + c, 0), side - 1);
-        for (int task = warp; task < nc * out_side; task += n_warps) {
-            const int ch = task / out_side, oy = task - ch * out_side;
-            const float sy = (oy + 0.5f) * ratio - 0.5f;
-            const int iy = (int)floorf(sy);
-            float wy[4];
-            cubic_weights(sy - (float)iy, wy);
+        for (int ch = warp; ch < nc; ch += n_warps) {
             const float* src = coarse + ch * stride;
-            float acc = 0.f;
-#pragma unroll
-            for (int a = 0; a < 4; ++a) {
-                const float* row = src + min(max(iy - 1 + a, 0), side - 1) * side;
-                float h = 0.f;                              // the row's four taps first, then its weight
+            auto hrow = [&](int r) -> float {
+                const float* row = src + min(max(r, 0), side - 1) * side;
+                float h = 0.f;
 #pragma unroll
                 for (int c = 0; c < 4; ++c) h = fmaf(wx[c], row[xx[c]], h);
-                acc = fmaf(wy[a], h, acc);
+                return h;
+            };
+            float* dst = xhat + ((long long)b * C + c0 + ch) * plane + ox;
+            int cur = -1000000;                             // source row of the window's second entry
+            float h0 = 0.f, h1 = 0.f, h2 = 0.f, h3 = 0.f;
+#pragma unroll 4
+            for (int oy = 0; oy < out_side; ++oy, dst += out_side) {
+                const int iy = row_src[oy];
+                const float4 wy = row_w[oy];
+                if (iy == cur + 1) {
+                    h0 = h1; h1 = h2; h2 = h3; h3 = hrow(iy + 2);
+                } else if (iy != cur) {
+                    h0 = hrow(iy - 1); h1 = hrow(iy); h2 = hrow(iy + 1); h3 = hrow(iy + 2);
+                }
+                cur = iy;
+                atomicAdd(dst, fmaf(wy.w, h3, fmaf(wy.z, h2, fmaf(wy.y, h1, wy.x * h0))));
             }
-            xhat[((long long)b * C + c0 + ch) * plane + (long long)oy * out_side + ox] += acc;
         }
     }
 }
@@ -145,7 +183,7 @@ hmar_recon_accumulate_staged_kernel(float* __restrict__ xhat, const float* __res
 cudaError_t launch_recon_accumulate(float* xhat, const float* codebook, const int* tokens_old, const int* tokens_new,
                                     const unsigned char* mask, int* tokens_out, int B, int C, int V, int side, int out_side,
                                     cudaStream_t stream) {
-    if (side <= kStageMaxSide) {
+    if (side <= kStageMaxSide && out_side <= kStageMaxOut) {
         const int n_groups = (C + kStageChannels - 1) / kStageChannels;
         {
             KernelTimer timer("hmar_recon_accumulate_kernel", stream);
