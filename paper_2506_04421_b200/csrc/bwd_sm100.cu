@@ -212,7 +212,12 @@ __device__ __forceinline__ int first_item_at_cost(const BwdArgs& args, long long
 // STRIDED: the bf16 tensors have the strides given in the arguments (packed projection layouts); otherwise they are
 // dense [BH, L, 64] and every address is formed with compile-time strides (the dense instantiation is the one the
 // benchmarks run: the extra address arithmetic and code of the strided one cost it a tenth of its speed).
-template <bool CHUNKED, bool STRIDED>
+// ONE_MASK: every tile goes through the variant of the softmax-gradient code with per-element bounds, so that the
+// block's code holds one variant instead of three.  It is the instantiation for side lists whose tiles are mostly
+// partial or packed (L = 680: 11 % faster, a third of the instruction-cache requests of the three-variant code
+// miss there); where most steps belong to full tiles the plain variant's shorter arithmetic wins (L = 2240: the
+// one-variant code is 4 % slower).
+template <bool CHUNKED, bool STRIDED, bool ONE_MASK>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                    const __grid_constant__ CUtensorMap map_v, const __grid_constant__ CUtensorMap map_do,
@@ -720,8 +725,8 @@ hmar_bwd_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             const BwdWork w = get_work(item_at(item, run));
             const int n_steps = steps_of(w);
             // the four key rows this thread works on in the softmax-gradient layout, and the queries that may see them
-            const bool tile_masked = (!w.uniform) || (w.row_count < BKV);
-            const bool rows_only = w.uniform != 0;          // only rows past the end of the tile are hidden
+            const bool tile_masked = ONE_MASK || (!w.uniform) || (w.row_count < BKV);
+            const bool rows_only = !ONE_MASK && w.uniform != 0;   // only rows past the end of the tile are hidden
             int qlo[4], qhi[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
@@ -866,14 +871,20 @@ static int sm_count() {
     return cached[dev];
 }
 
+// Side lists with fewer than this share (in thousandths) of their steps in full tiles run the one-variant
+// instantiation (L = 680 has 42 %, L = 2240 has 82 %).
+constexpr int kOneMaskBelowPermille = 600;
+
 template <bool STRIDED>
 static cudaError_t launch_bwd_tc_layout(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const CUtensorMap& dout_map,
                                         const CUtensorMap& dq_acc_map, const BwdArgs& args, const __nv_bfloat16* out,
                                         const __nv_bfloat16* dout, __nv_bfloat16* dq, int BH, cudaStream_t stream) {
     const size_t smem = sizeof(SharedStorage) + 1024;
-    cudaError_t e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<false, STRIDED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<false, STRIDED, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<true, STRIDED>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<true, STRIDED, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(hmar_bwd_tc_kernel<false, STRIDED, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const size_t n_rows = (size_t)BH * args.L;
     {
@@ -895,9 +906,11 @@ static cudaError_t launch_bwd_tc_layout(const CUtensorMap& q, const CUtensorMap&
             while (a.split > 0 && ((long long)BH * a.split + grid - 1) / grid > MAX_CHUNKS) a.split >>= 1;
         }
         if (a.split > 0)
-            hmar_bwd_tc_kernel<true, STRIDED><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
+            hmar_bwd_tc_kernel<true, STRIDED, false><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
+        else if (args.plain_permille < kOneMaskBelowPermille)
+            hmar_bwd_tc_kernel<false, STRIDED, true><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
         else
-            hmar_bwd_tc_kernel<false, STRIDED><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
+            hmar_bwd_tc_kernel<false, STRIDED, false><<<grid, NUM_THREADS, smem, stream>>>(q, k, v, dout_map, dq_acc_map, a);
     }
     const size_t n8 = n_rows * D / 8;
     {

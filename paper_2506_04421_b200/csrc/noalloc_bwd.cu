@@ -115,6 +115,7 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
         host_work[i].uniform = tiles[i].uniform;
     }
     const int head_cost = bwd_fill_costs(host_work, (int)tiles.size());
+    const int plain_permille = bwd_plain_permille(host_work, (int)tiles.size());
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     for (size_t first = 0; first < tiles.size(); first += kFillChunk) {
         WorkChunk chunk;
@@ -137,6 +138,7 @@ extern "C" int hmar_attn_bwd_noalloc(const void* q, const void* k, const void* v
     a.n_work = (int)tiles.size();
     a.n_heads = BH;
     a.head_cost = head_cost;
+    a.plain_permille = plain_permille;
     a.L = (int)L;
     a.scale_log2 = softmax_scale * 1.4426950408889634f;
     a.softmax_scale = softmax_scale;

@@ -52,11 +52,24 @@ inline int bwd_fill_costs(BwdWork* work, int n) {
     return acc;
 }
 
+// Share, in thousandths, of a head's steps that belong to full tiles (128 key rows that all see the whole query
+// range): those run without any mask code.
+inline int bwd_plain_permille(const BwdWork* work, int n) {
+    long long plain = 0, total = 0;
+    for (int i = 0; i < n; ++i) {
+        const int steps = (work[i].q_end - work[i].q_begin + 127) / 128;
+        total += steps;
+        if (work[i].uniform && work[i].row_count == 128) plain += steps;
+    }
+    return total > 0 ? (int)(plain * 1000 / total) : 1000;
+}
+
 struct BwdArgs {
     const BwdWork* work;
     int n_work;
     int n_heads;             // B * H
     int head_cost;           // from bwd_fill_costs
+    int plain_permille;      // from bwd_plain_permille: picks the instantiation of the main kernel
     int split;               // set by the launcher: runs per head dealt to the blocks in turn (0: one contiguous run per block)
     int L;
     float scale_log2;        // softmax_scale * log2(e)

@@ -76,6 +76,7 @@ struct Plan {
     int n_fwd = 0;
     int n_bwd = 0;
     int bwd_head_cost = 0;
+    int bwd_plain_permille = 1000;
     int zero_begin = 0, zero_end = 0;   // key rows of a head that no query sees: their dK, dV are zeros
 };
 
@@ -136,6 +137,7 @@ static const Plan* get_plan(const ScaleTable& st) {
     }
     static_assert(sizeof(FwdWork) == sizeof(BwdWork), "work tiles share one allocation");
     plan.bwd_head_cost = bwd_fill_costs(bwork.data(), (int)bwork.size());
+    plan.bwd_plain_permille = bwd_plain_permille(bwork.data(), (int)bwork.size());
     plan.n_fwd = (int)work.size();
     plan.n_bwd = (int)bwork.size();
     const size_t fwd_bytes = work.size() * sizeof(FwdWork), bwd_bytes = bwork.size() * sizeof(BwdWork);
@@ -280,6 +282,7 @@ static int tc_bwd_strided(const bf16* q, const bf16* k, const bf16* v, const bf1
     a.n_work = plan->n_bwd;
     a.n_heads = BH;
     a.head_cost = plan->bwd_head_cost;
+    a.plain_permille = plan->bwd_plain_permille;
     a.L = L;
     a.scale_log2 = scale * 1.4426950408889634f;
     a.softmax_scale = scale;
