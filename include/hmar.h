@@ -209,7 +209,9 @@ int hmar_attn_scale_step_strided(const void* q, const void* k_prev, const void* 
  *   tokens_new : [B, side, side] int32 ids, device;  tokens_old : the same shape, or NULL when mask is NULL
  *   mask       : [B, side, side] bytes, nonzero = take tokens_new there; NULL = take tokens_new everywhere
  *   tokens_out : [B, side, side] int32 or NULL; receives the selected map (must not alias the inputs)
- * side <= out_side <= 4096.  Ids outside [0, V) are clamped.  One kernel, asynchronous on `stream`. */
+ * side <= out_side <= 4096.  Ids outside [0, V) are clamped.  One kernel, asynchronous on `stream`; every
+ * element of xhat receives exactly one addition (issued as a reduction to memory), so the result does not
+ * depend on scheduling.  No alignment beyond the element types' own is required. */
 int hmar_recon_accumulate(float* xhat, const float* codebook, const int* tokens_old, const int* tokens_new,
                           const unsigned char* mask, int* tokens_out, int B, int C, int V, int side, int out_side,
                           void* stream);

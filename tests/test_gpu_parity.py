@@ -598,12 +598,14 @@ def test_repeat_calls_are_stable():
 
 
 @pytest.mark.parametrize("side,out_side,B,C,V", [(1, 32, 3, 32, 4096), (6, 32, 2, 32, 4096), (13, 32, 2, 32, 4096), (32, 32, 2, 32, 4096),
-                                                  (3, 7, 2, 5, 17), (16, 16, 65, 32, 4096), (5, 16, 2, 40, 33), (40, 48, 1, 8, 50)])
+                                                  (3, 7, 2, 5, 17), (16, 16, 65, 32, 4096), (5, 16, 2, 40, 33), (40, 48, 1, 8, 50),
+                                                  (8, 48, 2, 16, 100), (24, 64, 1, 8, 64), (8, 80, 1, 8, 30)])
 @pytest.mark.parametrize("masked", [False, True])
 def test_recon_accumulate_matches_oracle(side, out_side, B, C, V, masked):
     """The sampler's neighbour step (Alg. 2 lines 7-8 with the sub-step's token selection, Sec. 4.2) on a synthetic
     codebook: fp32 on the GPU against the fp64 oracle, and the selected token map bit for bit.  Maps of at most
-    32 x 32 tokens take the staged kernel (also with more than 32 channels), the 40 x 40 case the plain one."""
+    32 x 32 tokens and reconstructions of at most 64 x 64 take the staged kernel (also with more than 32 channels,
+    and with more than 32 output columns), the 40 x 40 map and the 80 x 80 reconstruction the plain one."""
     rng = np.random.default_rng(1000 * side + out_side + int(masked))
     codebook = rng.standard_normal((V, C)).astype(np.float32)
     old = rng.integers(0, V, (B, side, side)).astype(np.int32)
@@ -622,6 +624,25 @@ def test_recon_accumulate_matches_oracle(side, out_side, B, C, V, masked):
     err = np.abs(xhat.double().cpu().numpy() - ref)
     assert err.max() <= 1e-5 * max(1.0, np.abs(ref).max()), f"max abs err {err.max():.3e}"
     assert all(intact() for intact in guards)
+
+
+def test_recon_accumulate_codebook_off_16_byte_alignment():
+    """A codebook whose base address is not a multiple of 16 bytes takes the staged kernel's one-value-at-a-time
+    gather; same result as the oracle."""
+    rng = np.random.default_rng(77)
+    V, C, side, out_side, B = 40, 8, 6, 16, 2
+    codebook = rng.standard_normal((V, C)).astype(np.float32)
+    new = rng.integers(0, V, (B, side, side)).astype(np.int32)
+    x0 = rng.standard_normal((B, C, out_side, out_side)).astype(np.float32)
+    buf = torch.zeros(V * C + 1, dtype=torch.float32, device="cuda")
+    cb = buf[1:].view(V, C)
+    cb.copy_(torch.from_numpy(codebook))
+    assert cb.data_ptr() % 16 == 4
+    xhat = torch.from_numpy(x0).cuda()
+    hmar.hmar_recon_accumulate(xhat, cb, torch.from_numpy(new).cuda())
+    ref = orc.recon_accumulate(x0, codebook, new, out_side)
+    err = np.abs(xhat.double().cpu().numpy() - ref)
+    assert err.max() <= 1e-5 * max(1.0, np.abs(ref).max()), f"max abs err {err.max():.3e}"
 
 
 def test_edge_cases_through_the_checking_build():
