@@ -660,7 +660,9 @@ def _finish(args, wl, world, rank, dev, total_ms, e2e_ms, fwd_ms, bwd_ms, launch
 def run_case(args):
     """A named side case run a few times (for profiling one kernel on a workload that is not the headline's):
     `256_d30_train` = forward + backward of the L = 680 training config at its full batch; `infer_scale7` = the
-    inference step of scale 7 (169 queries, 250 keys) at B = 64, H = 24.  Prints a small JSON line."""
+    inference step of scale 7 (169 queries, 250 keys) at B = 64, H = 24; `recon_b2048` = the sampler's neighbour step
+    on a 32 x 32 x 32 reconstruction at B = 2048 (268 MB), a 13 x 13 map then the 32 x 32 one per repetition.
+    Prints a small JSON line."""
     import torch
 
     import paper_2506_04421_b200 as hmar
@@ -676,6 +678,19 @@ def run_case(args):
         for _ in range(args.warmup + reps):
             out, lse = hmar.hmar_attn_fwd(q, k, v, wl_x.side_lens, wl_x.softmax_scale)
             hmar.hmar_attn_bwd(q, k, v, out, lse, do, wl_x.side_lens, wl_x.softmax_scale)
+    elif args.case == "recon_b2048":
+        g = torch.Generator(device=dev)
+        g.manual_seed(4421)
+        V, C, S, B = 4096, 32, 32, 2048
+        codebook = torch.randn((V, C), generator=g, device=dev)
+        xhat = torch.zeros((B, C, S, S), device=dev)
+        maps = {side: [torch.randint(0, V, (B, side, side), generator=g, device=dev, dtype=torch.int32) for _ in range(2)] +
+                      [torch.randint(0, 2, (B, side, side), generator=g, device=dev, dtype=torch.uint8),
+                       torch.empty((B, side, side), device=dev, dtype=torch.int32)] for side in (13, 32)}
+        for _ in range(args.warmup + reps):
+            for side in (13, 32):
+                new, old, mask, sel = maps[side]
+                hmar.hmar_recon_accumulate(xhat, codebook, new, old, mask, sel)
     else:
         wl_x = CONFIGS["512_d24_infer"]
         s_ = 6
@@ -696,7 +711,7 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--batch", type=int, default=0,
                     help="override the batch size (profiling on a reduced case; named in config.workload)")
-    ap.add_argument("--case", choices=["256_d30_train", "infer_scale7"], default=None,
+    ap.add_argument("--case", choices=["256_d30_train", "infer_scale7", "recon_b2048"], default=None,
                     help="run a named side case a few times instead of the benchmark (profiling)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline leg")
