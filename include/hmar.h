@@ -229,6 +229,13 @@ int hmar_schedule_tiles(int n_scales, const int* side_lens, int direction,
 int hmar_schedule_tiles_window(int n_scales, const int* side_lens, int window, int direction,
                                int32_t* tiles, int max_tiles);
 
+/* Share, in thousandths, of a head's backward steps (128 key rows x 128 query rows) that belong to full tiles:
+ * 128 key rows that all see the tile's whole query range, which the backward kernel processes without mask code.
+ * The backward picks its instantiation by it: side lists below 600 run the one that keeps a single, fully
+ * masked variant of the softmax-gradient code (smaller code; these lists are bound by instruction fetch), the
+ * others the one with three variants.  Returns a negative hmar_status for a bad side list.  Host only. */
+int hmar_schedule_bwd_full_tile_share(int n_scales, const int* side_lens, int window);
+
 /* Blocks until the work queued on the current device has finished, then returns the code recorded
  * by the kernels since the last call (HMAR_OK, or HMAR_ERR_DEVICE_TIMEOUT with *detail, if not NULL,
  * telling which wait gave up) and clears it.

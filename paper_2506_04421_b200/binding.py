@@ -30,7 +30,7 @@ HMAR_WINDOW_PREV = 3        # scale k-1 only; the first scale attends to itself
 EXPORTED_SYMBOLS = (
     "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_fwd_window", "hmar_attn_fwd_window_f32", "hmar_attn_fwd_packed", "hmar_attn_bwd_packed",
     "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd", "hmar_attn_bwd_f32", "hmar_attn_bwd_window",
-    "hmar_attn_bwd_window_f32", "hmar_schedule_tiles_window", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_attn_scale_step_strided", "hmar_schedule_tiles",
+    "hmar_attn_bwd_window_f32", "hmar_schedule_tiles_window", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_attn_scale_step_strided", "hmar_schedule_tiles", "hmar_schedule_bwd_full_tile_share",
     "hmar_recon_accumulate", "hmar_device_status", "hmar_selftest_bounded_wait", "hmar_profile_begin", "hmar_profile_end", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
     "hmar_status_string",
 )
@@ -69,6 +69,7 @@ def lib():
     L.hmar_attn_bwd_window.argtypes = [vp] * 9 + [vp, ctypes.c_size_t, i, i, i, i, ip, i, fp, vp]
     L.hmar_attn_bwd_window_f32.argtypes = L.hmar_attn_bwd_window.argtypes
     L.hmar_schedule_tiles_window.argtypes = [i, ip, i, i, ctypes.POINTER(ctypes.c_int32), i]
+    L.hmar_schedule_bwd_full_tile_share.argtypes = [i, ip, i]
     L.hmar_attn_bwd_noalloc.argtypes = [vp] * 9 + [i, i, i, i, ip, fp, vp]
     L.hmar_attn_scale_step.argtypes = [vp] * 7 + [i, i, i, i, i, fp, vp]
     L.hmar_attn_scale_step_f32.argtypes = L.hmar_attn_scale_step.argtypes
@@ -304,6 +305,15 @@ def hmar_schedule_tiles(side_lens, direction, window=HMAR_WINDOW_MARKOV):
     lib().hmar_schedule_tiles_window(n, sides, int(window), int(direction), buf, count)
     keys = ("row_begin", "row_count", "partner_begin", "partner_end", "uniform", "cost")
     return [dict(zip(keys, buf[6 * t:6 * t + 6])) for t in range(count)]
+
+
+def hmar_schedule_bwd_full_tile_share(side_lens, window=HMAR_WINDOW_MARKOV):
+    """Thousandths of a head's backward steps that lie in full tiles (host only; needs no GPU)."""
+    sides, n = _sides(side_lens)
+    share = lib().hmar_schedule_bwd_full_tile_share(n, sides, int(window))
+    if share < 0:
+        raise HmarError(share, "hmar_schedule_bwd_full_tile_share")
+    return share
 
 
 def hmar_device_status():

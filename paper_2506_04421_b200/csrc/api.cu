@@ -362,6 +362,13 @@ int hmar_schedule_tiles_window(int n_scales, const int* side_lens, int window, i
     return (int)t.size();
 }
 
+int hmar_schedule_bwd_full_tile_share(int n_scales, const int* side_lens, int window) {
+    ScaleTable st;
+    int rc = check_sides(n_scales, side_lens, window, &st);
+    if (rc != HMAR_OK) return rc;
+    return tc_bwd_full_tile_permille(st);
+}
+
 int hmar_device_status(int* detail) {
     if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return HMAR_ERR_CUDA; }
     int host[2] = {0, 0};

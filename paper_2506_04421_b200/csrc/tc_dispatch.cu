@@ -91,6 +91,38 @@ struct PlanKey {
 static std::mutex g_plan_mu;
 static std::map<PlanKey, Plan> g_plans;
 
+// The backward's work list of one head: a tile of 128 key rows each, with the query range that may see it.
+// Key tiles that no query sees (the last scale under HMAR_WINDOW_PREV) are not work items: the backward
+// kernel's pipeline wants at least one step per item.  Their rows are one stretch at the end of the head,
+// returned in [zero_begin, zero_end) (their dK, dV are zeros).
+static std::vector<BwdWork> make_bwd_work(const ScaleTable& st, int& zero_begin, int& zero_end) {
+    std::vector<Tile> btiles = build_tiles(st, 1);
+    std::vector<Tile> live;
+    zero_begin = zero_end = 0;
+    for (const Tile& t : btiles) {
+        if (t.partner_end > t.partner_begin) { live.push_back(t); continue; }
+        if (zero_end == zero_begin) { zero_begin = t.row_begin; zero_end = t.row_begin + t.row_count; }
+        zero_begin = std::min(zero_begin, (int)t.row_begin);
+        zero_end = std::max(zero_end, (int)(t.row_begin + t.row_count));
+    }
+    std::vector<BwdWork> bwork(live.size());
+    for (size_t i = 0; i < live.size(); ++i) {
+        bwork[i] = BwdWork{};
+        bwork[i].row_begin = live[i].row_begin;
+        bwork[i].row_count = live[i].row_count;
+        bwork[i].q_begin = live[i].partner_begin;
+        bwork[i].q_end = live[i].partner_end;
+        bwork[i].uniform = live[i].uniform;
+    }
+    return bwork;
+}
+
+int tc_bwd_full_tile_permille(const ScaleTable& st) {
+    int zb = 0, ze = 0;
+    std::vector<BwdWork> bwork = make_bwd_work(st, zb, ze);
+    return bwd_plain_permille(bwork.data(), (int)bwork.size());
+}
+
 static const Plan* get_plan(const ScaleTable& st) {
     PlanKey key;
     if (cudaGetDevice(&key.device) != cudaSuccess) return nullptr;
@@ -111,30 +143,8 @@ static const Plan* get_plan(const ScaleTable& st) {
         work[i].uniform = tiles[i].uniform;
         work[i].pad = 0;
     }
-    std::vector<Tile> btiles = build_tiles(st, 1);
-    // Key tiles that no query sees (the last scale under HMAR_WINDOW_PREV) are not work items: the backward
-    // kernel's pipeline wants at least one step per item.  Their rows are one stretch at the end of the head.
     Plan plan;
-    {
-        std::vector<Tile> live;
-        plan.zero_begin = plan.zero_end = 0;
-        for (const Tile& t : btiles) {
-            if (t.partner_end > t.partner_begin) { live.push_back(t); continue; }
-            if (plan.zero_end == plan.zero_begin) { plan.zero_begin = t.row_begin; plan.zero_end = t.row_begin + t.row_count; }
-            plan.zero_begin = std::min(plan.zero_begin, (int)t.row_begin);
-            plan.zero_end = std::max(plan.zero_end, (int)(t.row_begin + t.row_count));
-        }
-        btiles.swap(live);
-    }
-    std::vector<BwdWork> bwork(btiles.size());
-    for (size_t i = 0; i < btiles.size(); ++i) {
-        bwork[i] = BwdWork{};
-        bwork[i].row_begin = btiles[i].row_begin;
-        bwork[i].row_count = btiles[i].row_count;
-        bwork[i].q_begin = btiles[i].partner_begin;
-        bwork[i].q_end = btiles[i].partner_end;
-        bwork[i].uniform = btiles[i].uniform;
-    }
+    std::vector<BwdWork> bwork = make_bwd_work(st, plan.zero_begin, plan.zero_end);
     static_assert(sizeof(FwdWork) == sizeof(BwdWork), "work tiles share one allocation");
     plan.bwd_head_cost = bwd_fill_costs(bwork.data(), (int)bwork.size());
     plan.bwd_plain_permille = bwd_plain_permille(bwork.data(), (int)bwork.size());

@@ -14,6 +14,8 @@ int tc_bwd(const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* 
            const float* lse, const __nv_bfloat16* dout, __nv_bfloat16* dq, __nv_bfloat16* dk,
            __nv_bfloat16* dv, float* delta, float* dq_acc, int BH, const ScaleTable& st, float scale,
            int* status, cudaStream_t stream);
+// Share (thousandths) of a head's backward steps that lie in full tiles; picks the main kernel's instantiation.  Host only.
+int tc_bwd_full_tile_permille(const ScaleTable& st);
 int tc_bwd_packed(const __nv_bfloat16* qkv, const __nv_bfloat16* out, const float* lse, const __nv_bfloat16* dout,
                   __nv_bfloat16* dqkv, float* delta, float* dq_acc, int B, int H, const ScaleTable& st, float scale,
                   int* status, cudaStream_t stream);

@@ -164,3 +164,29 @@ def test_prev_window_backward_tiles_leave_out_nothing_but_the_last_scale():
         assert all(t["row_begin"] >= last_begin for t in empty)
         covered = sum(t["row_count"] for t in empty)
         assert covered <= sides[-1] ** 2
+
+
+def test_backward_full_tile_share_picks_the_instantiation():
+    """The share of a head's backward steps in full tiles, recomputed here from the exported tile list, and on
+    which side of the 60 % line the paper's two training resolutions fall (Sec. 5: 256 x 256 has L = 680,
+    512 x 512 has L = 2240): the short list runs the one-variant backward, the long one the three-variant one."""
+    def share(side_lens, window=hmar.HMAR_WINDOW_MARKOV):
+        plain = total = 0
+        for t in hmar.hmar_schedule_tiles(side_lens, 1, window=window):
+            steps = (t["partner_end"] - t["partner_begin"] + 127) // 128
+            total += steps
+            if t["uniform"] and t["row_count"] == 128:
+                plain += steps
+        return plain * 1000 // total
+    short, long_ = CONFIGS["256_d30_train"].side_lens, CONFIGS["512_d24_train"].side_lens
+    for sides in (short, long_, (1, 2), (16, 16), (12, 12, 12)):
+        assert hmar.hmar_schedule_bwd_full_tile_share(sides) == share(sides), sides
+    for window in (hmar.HMAR_WINDOW_CAUSAL, hmar.HMAR_WINDOW_SELF, hmar.HMAR_WINDOW_PREV):
+        assert hmar.hmar_schedule_bwd_full_tile_share(long_, window) == share(long_, window)
+    assert hmar.hmar_schedule_bwd_full_tile_share(short) < 600 <= hmar.hmar_schedule_bwd_full_tile_share(long_)
+    # (16, 16): four full tiles of 128 keys (two per scale), seen by 512 and by 256 queries: every step is plain
+    assert hmar.hmar_schedule_bwd_full_tile_share((16, 16)) == 1000
+    # (1, 2): one packed tile of 5 key rows, never full
+    assert hmar.hmar_schedule_bwd_full_tile_share((1, 2)) == 0
+    with pytest.raises(hmar.HmarError):
+        hmar.hmar_schedule_bwd_full_tile_share((1, 0))
