@@ -225,3 +225,26 @@ def recon_accumulate(xhat, codebook, tokens, out_side):
     looked = codebook[tokens]                                   # [B, side, side, C]
     coarse = np.moveaxis(looked, -1, 1)                         # [B, C, side, side]
     return np.asarray(xhat, dtype=np.float64) + bicubic_upsample(coarse, out_side)
+
+
+def area_downsample(x, out_side):
+    """The running reconstruction brought down to a scale's resolution (Sec. 4.1: the interpolation of Alg. 1's
+    loop maps x~_{1:k-1} to an H_k x W_k image, which the scale is conditioned on).  The paper does not name the
+    interpolation; reading used here, the counterpart of the bicubic enlargement above in the VAR tokenizer family:
+    area interpolation, i.e. output pixel (i, j) is the plain mean of the input pixels whose rows lie in
+    [floor(i * h / out), ceil((i + 1) * h / out)) and whose columns lie in the like range.
+
+    x: [..., h, w] float64 -> [..., out_side, out_side]; out_side <= h, w."""
+    x = np.asarray(x, dtype=np.float64)
+    h, w = x.shape[-2], x.shape[-1]
+    out = np.zeros(x.shape[:-2] + (out_side, out_side), dtype=np.float64)
+    for i in range(out_side):
+        r0, r1 = (i * h) // out_side, -((-(i + 1) * h) // out_side)
+        for j in range(out_side):
+            c0, c1 = (j * w) // out_side, -((-(j + 1) * w) // out_side)
+            acc = 0.0
+            for r in range(r0, r1):
+                for c in range(c0, c1):
+                    acc = acc + x[..., r, c]
+            out[..., i, j] = acc / ((r1 - r0) * (c1 - c0))
+    return out

@@ -631,3 +631,37 @@ def test_pins_detect_planted_mistakes_in_the_added_functions(monkeypatch):
     good_acc = orc.recon_accumulate
     monkeypatch.setattr(orc, "recon_accumulate", lambda x, cb, t, s: good_acc(np.zeros_like(np.asarray(x, dtype=np.float64)), cb, t, s))
     assert fails(test_select_tokens_and_recon_accumulate)
+
+
+def test_area_downsample_against_the_library_routine_closed_forms_and_a_planted_mistake():
+    """Pins of the oracle's area interpolation: the library's routine in fp64, block means where the sizes divide,
+    a hand-computed 3 -> 2 case (bins {0, 1} and {1, 2}), identity, constants, the global mean at size 1, and a
+    planted mistake (ceil taken as floor for the bin's end) that the library comparison catches."""
+    rng = np.random.default_rng(35)
+    for h, s in ((32, 1), (32, 13), (32, 16), (32, 32), (16, 6), (7, 3), (9, 4), (64, 24), (5, 5)):
+        x = rng.standard_normal((2, 3, h, h))
+        ref = torch.nn.functional.interpolate(torch.from_numpy(x), size=(s, s), mode="area").numpy()
+        np.testing.assert_allclose(orc.area_downsample(x, s), ref, rtol=1e-12, atol=1e-13)
+    x = rng.standard_normal((3, 12, 12))
+    np.testing.assert_allclose(orc.area_downsample(x, 4), x.reshape(3, 4, 3, 4, 3).mean(axis=(2, 4)), rtol=1e-13)   # block means
+    np.testing.assert_allclose(orc.area_downsample(x, 1)[:, 0, 0], x.mean(axis=(1, 2)), rtol=1e-13)
+    assert np.array_equal(orc.area_downsample(x, 12), x)
+    np.testing.assert_allclose(orc.area_downsample(np.full((9, 9), -1.25), 4), -1.25, rtol=1e-15)
+    y = np.arange(9.0).reshape(3, 3)          # rows {0,1} / {1,2} and the like columns
+    np.testing.assert_allclose(orc.area_downsample(y, 2), [[(0 + 1 + 3 + 4) / 4, (1 + 2 + 4 + 5) / 4],
+                                                           [(3 + 4 + 6 + 7) / 4, (4 + 5 + 7 + 8) / 4]], rtol=1e-15)
+    np.testing.assert_allclose(orc.area_downsample(y.T, 2), orc.area_downsample(y, 2).T, rtol=1e-15)
+
+    def planted(x, s):                        # end of the bin rounded down: drops the shared row / column
+        h = x.shape[-1]
+        out = np.zeros(x.shape[:-2] + (s, s))
+        for i in range(s):
+            r0, r1 = (i * h) // s, max(((i + 1) * h) // s, (i * h) // s + 1)
+            for j in range(s):
+                c0, c1 = (j * h) // s, max(((j + 1) * h) // s, (j * h) // s + 1)
+                out[..., i, j] = x[..., r0:r1, c0:c1].mean(axis=(-2, -1))
+        return out
+    z = rng.standard_normal((7, 7))
+    ref = torch.nn.functional.interpolate(torch.from_numpy(z)[None, None], size=(3, 3), mode="area").numpy()[0, 0]
+    assert np.abs(planted(z, 3) - ref).max() > 1e-3
+    np.testing.assert_allclose(orc.area_downsample(z, 3), ref, rtol=1e-12, atol=1e-13)
