@@ -254,7 +254,9 @@ def time_recon(hmar, dev, peaks, reps=20):
     """The sampler's neighbour step (Alg. 2 lines 7-8 fused with the sub-step's token selection) on a synthetic
     codebook (V = 4096, C = 32), latent 32 x 32: at the sampler's batch (64) and at a batch whose reconstruction
     exceeds L2 (2048: 268 MB), for the last scale (32 -> 32) and a middle one (13 -> 32).  GB/s on the algorithmic
-    bytes (the reconstruction read and written once) against the measured HBM bandwidth."""
+    bytes (the reconstruction read and written once) against the measured HBM bandwidth.  Then the other neighbour,
+    the area interpolation of the reconstruction down to those two sizes (Sec. 4.1; algorithmic bytes: the
+    reconstruction read once plus the small image written)."""
     import torch
     rows = []
     g = torch.Generator(device=dev)
@@ -278,7 +280,21 @@ def time_recon(hmar, dev, peaks, reps=20):
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1) / reps
             byt = 2 * xhat.numel() * 4
-            rows.append({"B": B, "side": side, "ms": round(ms, 4), "gbs": round(byt / ms / 1e6, 1),
+            rows.append({"op": "accumulate", "B": B, "side": side, "ms": round(ms, 4), "gbs": round(byt / ms / 1e6, 1),
+                         "frac_hbm": round(byt / ms / 1e6 / peaks["hbm_gbs"], 4), "algorithmic_bytes": byt})
+        for side in (13, 32):                              # the other neighbour: area interpolation down to a scale
+            out = torch.empty((B, C, side, side), device=dev)
+            for _ in range(3):
+                hmar.hmar_recon_downsample(xhat, side, out=out)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                hmar.hmar_recon_downsample(xhat, side, out=out)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / reps
+            byt = (xhat.numel() + out.numel()) * 4
+            rows.append({"op": "downsample", "B": B, "side": side, "ms": round(ms, 4), "gbs": round(byt / ms / 1e6, 1),
                          "frac_hbm": round(byt / ms / 1e6 / peaks["hbm_gbs"], 4), "algorithmic_bytes": byt})
         del xhat
         torch.cuda.empty_cache()

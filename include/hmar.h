@@ -216,6 +216,15 @@ int hmar_recon_accumulate(float* xhat, const float* codebook, const int* tokens_
                           const unsigned char* mask, int* tokens_out, int B, int C, int V, int side, int out_side,
                           void* stream);
 
+/* The other sampler-side step (Sec. 4.1, "Reformulating Next-Scale Prediction to be Markovian": the running
+ * reconstruction x~_{1:k-1} is interpolated to the scale's resolution, and the scale is conditioned on that
+ * image instead of on all earlier token maps).  The paper does not name the interpolation; this is area
+ * interpolation: out(i, j) = the mean of xhat over rows [floor(i * in_side / out_side),
+ * ceil((i + 1) * in_side / out_side)) and the like columns.
+ *   xhat : [B, C, in_side, in_side] fp32, device (read only);  out : [B, C, out_side, out_side] fp32, device
+ * out_side <= in_side <= 4096; the buffers must not overlap.  One kernel, asynchronous on `stream`. */
+int hmar_recon_downsample(const float* xhat, float* out, int B, int C, int in_side, int out_side, void* stream);
+
 /* Host-side scale-block scheduler (Sec. 4.1: the kernel visits only the live blocks of the mask).
  * Writes the work list of one head for `direction` 0 = forward (tiles of query rows, each with the
  * contiguous key range it must visit) or 1 = backward (tiles of key rows with their query range).

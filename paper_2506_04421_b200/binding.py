@@ -31,7 +31,7 @@ EXPORTED_SYMBOLS = (
     "hmar_attn_fwd", "hmar_attn_fwd_f32", "hmar_attn_fwd_window", "hmar_attn_fwd_window_f32", "hmar_attn_fwd_packed", "hmar_attn_bwd_packed",
     "hmar_attn_bwd_workspace_bytes", "hmar_attn_bwd", "hmar_attn_bwd_f32", "hmar_attn_bwd_window",
     "hmar_attn_bwd_window_f32", "hmar_schedule_tiles_window", "hmar_attn_bwd_noalloc", "hmar_attn_scale_step", "hmar_attn_scale_step_f32", "hmar_attn_scale_step_strided", "hmar_schedule_tiles", "hmar_schedule_bwd_full_tile_share",
-    "hmar_recon_accumulate", "hmar_device_status", "hmar_selftest_bounded_wait", "hmar_profile_begin", "hmar_profile_end", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
+    "hmar_recon_accumulate", "hmar_recon_downsample", "hmar_device_status", "hmar_selftest_bounded_wait", "hmar_profile_begin", "hmar_profile_end", "hmar_debug_force_simt", "hmar_launch_count", "hmar_shutdown",
     "hmar_status_string",
 )
 
@@ -77,6 +77,7 @@ def lib():
     L.hmar_attn_scale_step_strided.argtypes = [vp] * 7 + [i, i, i, i, i, ll, ll, ll, ll, fp, vp]
     L.hmar_schedule_tiles.argtypes = [i, ip, i, ctypes.POINTER(ctypes.c_int32), i]
     L.hmar_recon_accumulate.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, i, vp]
+    L.hmar_recon_downsample.argtypes = [vp, vp, i, i, i, i, vp]
     L.hmar_device_status.argtypes = [ip]
     L.hmar_selftest_bounded_wait.argtypes = [vp]
     L.hmar_profile_begin.restype = None
@@ -293,6 +294,20 @@ def hmar_recon_accumulate(xhat, codebook, tokens_new, tokens_old=None, mask=None
     _check(lib().hmar_recon_accumulate(_ptr(xhat), _ptr(codebook), _ptr(tokens_old), _ptr(tokens_new), _ptr(mask),
                                        _ptr(tokens_out), B, C, V, side, S, _stream(stream)), "hmar_recon_accumulate")
     return xhat
+
+
+def hmar_recon_downsample(xhat, out_side, out=None, stream=None):
+    """Area interpolation of xhat [B,C,S,S] fp32 down to [B,C,out_side,out_side]; returns the result."""
+    _need(xhat, out)
+    if xhat.dtype != torch.float32:
+        raise TypeError("xhat must be float32")
+    B, C, S, _ = xhat.shape
+    if out is None:
+        out = torch.empty((B, C, out_side, out_side), dtype=torch.float32, device=xhat.device)
+    elif out.dtype != torch.float32 or tuple(out.shape) != (B, C, out_side, out_side):
+        raise ValueError("out must be float32 [B, C, out_side, out_side]")
+    _check(lib().hmar_recon_downsample(_ptr(xhat), _ptr(out), B, C, S, int(out_side), _stream(stream)), "hmar_recon_downsample")
+    return out
 
 
 def hmar_schedule_tiles(side_lens, direction, window=HMAR_WINDOW_MARKOV):

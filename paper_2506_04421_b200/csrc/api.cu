@@ -432,6 +432,16 @@ int hmar_recon_accumulate(float* xhat, const float* codebook, const int* tokens_
                                    static_cast<cudaStream_t>(stream)) == cudaSuccess ? HMAR_OK : HMAR_ERR_CUDA;
 }
 
+int hmar_recon_downsample(const float* xhat, float* out, int B, int C, int in_side, int out_side, void* stream) {
+    if (B <= 0 || C <= 0 || in_side <= 0 || out_side <= 0 || in_side > 4096 || C > 4096) return HMAR_ERR_BAD_ARG;
+    if (out_side > in_side) return HMAR_ERR_BAD_ARG;                    // the step only ever shrinks the image
+    if (xhat == nullptr || out == nullptr || xhat == out) return HMAR_ERR_BAD_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return HMAR_ERR_CUDA; }
+    return launch_recon_downsample(xhat, out, B, C, in_side, out_side, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? HMAR_OK : HMAR_ERR_CUDA;
+}
+
 int hmar_selftest_bounded_wait(void* stream) {
     int rc = check_device();
     if (rc != HMAR_OK) return rc;

@@ -34,5 +34,7 @@ cudaError_t simt_bwd(const T* q, const T* k, const T* v, const T* out, const flo
 cudaError_t launch_recon_accumulate(float* xhat, const float* codebook, const int* tokens_old, const int* tokens_new,
                                     const unsigned char* mask, int* tokens_out, int B, int C, int V, int side, int out_side,
                                     cudaStream_t stream);
+cudaError_t launch_recon_downsample(const float* xhat, float* out, int B, int C, int in_side, int out_side,
+                                    cudaStream_t stream);
 
 }  // namespace hmar

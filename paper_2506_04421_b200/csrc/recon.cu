@@ -178,6 +178,75 @@ hmar_recon_accumulate_staged_kernel(float* __restrict__ xhat, const float* __res
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The running reconstruction brought down to a scale's resolution (Sec. 4.1: the scale is conditioned on the
+// interpolated x~_{1:k-1}): area interpolation, out(i, j) = mean of the input over rows
+// [floor(i * S / s), ceil((i + 1) * S / s)) and the like columns.
+//
+// Staged kernel: a warp per image plane.  The plane is read once, coalesced, into shared memory (rows padded by
+// one word); lane = input row sums the row's column bins (partial sums, row stride odd so the lanes hit
+// different banks); lane = output column sums those over the row bins, divides by the bin's size and writes
+// a coalesced output row.  One read of the reconstruction, which is all the traffic that counts.
+__device__ __forceinline__ int bin_begin(int i, int in, int out) { return (i * in) / out; }
+__device__ __forceinline__ int bin_end(int i, int in, int out) { return ((i + 1) * in + out - 1) / out; }
+
+__global__ void __launch_bounds__(256)
+hmar_recon_downsample_staged_kernel(const float* __restrict__ xhat, float* __restrict__ out, long long n_planes,
+                                    int S, int s, int warps_per_block) {
+    extern __shared__ float down_smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ts = s | 1;                                   // row stride of the partial sums
+    const int per_warp = S * (S + 1) + S * ts;
+    float* tile = down_smem + warp * per_warp;
+    float* part = tile + S * (S + 1);
+    const long long plane = (long long)blockIdx.x * warps_per_block + warp;
+    if (warp >= warps_per_block || plane >= n_planes) return;
+    const float* src = xhat + plane * S * S;
+    for (int i = lane; i < S * S; i += 32) {
+        const int r = i / S, c = i - r * S;
+        tile[r * (S + 1) + c] = src[i];
+    }
+    __syncwarp();
+    for (int r = lane; r < S; r += 32) {
+        const float* row = tile + r * (S + 1);
+        for (int ox = 0; ox < s; ++ox) {
+            const int c0 = bin_begin(ox, S, s), c1 = bin_end(ox, S, s);
+            float acc = 0.f;
+            for (int c = c0; c < c1; ++c) acc += row[c];
+            part[r * ts + ox] = acc;
+        }
+    }
+    __syncwarp();
+    float* dst = out + plane * s * s;
+    for (int ox = lane; ox < s; ox += 32) {
+        const int nc = bin_end(ox, S, s) - bin_begin(ox, S, s);
+        for (int oy = 0; oy < s; ++oy) {
+            const int r0 = bin_begin(oy, S, s), r1 = bin_end(oy, S, s);
+            float acc = 0.f;
+            for (int r = r0; r < r1; ++r) acc += part[r * ts + ox];
+            dst[oy * s + ox] = acc / (float)((r1 - r0) * nc);
+        }
+    }
+}
+
+// Plain kernel for planes too large to stage: a thread per output pixel sums its bin from global memory.
+__global__ void __launch_bounds__(256)
+hmar_recon_downsample_kernel(const float* __restrict__ xhat, float* __restrict__ out, long long n_out, int S, int s) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n_out) return;
+    const int ox = (int)(idx % s), oy = (int)((idx / s) % s);
+    const long long plane = idx / ((long long)s * s);
+    const int r0 = bin_begin(oy, S, s), r1 = bin_end(oy, S, s), c0 = bin_begin(ox, S, s), c1 = bin_end(ox, S, s);
+    const float* src = xhat + plane * S * S;
+    float acc = 0.f;
+    for (int r = r0; r < r1; ++r) {
+        float row = 0.f;
+        for (int c = c0; c < c1; ++c) row += __ldg(src + (long long)r * S + c);
+        acc += row;
+    }
+    out[idx] = acc / (float)((r1 - r0) * (c1 - c0));
+}
+
 }  // namespace
 
 cudaError_t launch_recon_accumulate(float* xhat, const float* codebook, const int* tokens_old, const int* tokens_new,
@@ -199,6 +268,37 @@ cudaError_t launch_recon_accumulate(float* xhat, const float* codebook, const in
         KernelTimer timer("hmar_recon_accumulate_kernel", stream);
         hmar_recon_accumulate_kernel<<<grid, 256, 0, stream>>>(xhat, codebook, tokens_old, tokens_new, mask, tokens_out, B, C, V,
                                                               side, out_side);
+    }
+    count_launch(1);
+    return cudaGetLastError();
+}
+
+constexpr int kDownStageMaxSide = 64;
+constexpr size_t kDownStageSmem = 96 * 1024;
+
+cudaError_t launch_recon_downsample(const float* xhat, float* out, int B, int C, int in_side, int out_side,
+                                    cudaStream_t stream) {
+    const long long n_planes = (long long)B * C;
+    if (in_side <= kDownStageMaxSide) {
+        const size_t per_warp = ((size_t)in_side * (in_side + 1) + (size_t)in_side * (out_side | 1)) * sizeof(float);
+        int warps = (int)(kDownStageSmem / per_warp);
+        warps = warps > 8 ? 8 : warps;                      // >= 2 at the largest staged plane
+        const size_t smem = per_warp * warps;
+        cudaError_t e = cudaFuncSetAttribute(hmar_recon_downsample_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kDownStageSmem);
+        if (e != cudaSuccess) return e;
+        {
+            KernelTimer timer("hmar_recon_downsample_kernel", stream);
+            hmar_recon_downsample_staged_kernel<<<(unsigned)((n_planes + warps - 1) / warps), 256, smem, stream>>>(
+                xhat, out, n_planes, in_side, out_side, warps);
+        }
+        count_launch(1);
+        return cudaGetLastError();
+    }
+    const long long n_out = n_planes * out_side * out_side;
+    {
+        KernelTimer timer("hmar_recon_downsample_kernel", stream);
+        hmar_recon_downsample_kernel<<<(unsigned)((n_out + 255) / 256), 256, 0, stream>>>(xhat, out, n_out, in_side, out_side);
     }
     count_launch(1);
     return cudaGetLastError();

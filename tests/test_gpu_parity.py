@@ -626,6 +626,26 @@ def test_recon_accumulate_matches_oracle(side, out_side, B, C, V, masked):
     assert all(intact() for intact in guards)
 
 
+@pytest.mark.parametrize("S,s,B,C", [(32, 1, 3, 5), (32, 13, 2, 32), (32, 16, 9, 8), (32, 32, 2, 4), (16, 6, 2, 7), (7, 3, 1, 3),
+                                     (64, 24, 2, 3), (64, 64, 1, 2), (80, 9, 1, 2), (5, 5, 1, 1)])
+def test_recon_downsample_matches_oracle(S, s, B, C):
+    """The running reconstruction brought down to a scale's resolution (Sec. 4.1) by area interpolation: fp32 on the
+    GPU against the fp64 oracle.  Planes of at most 64 x 64 take the staged kernel, the 80 x 80 case the plain one;
+    the output sits between canaries."""
+    rng = np.random.default_rng(100 * S + s)
+    x = rng.standard_normal((B, C, S, S)).astype(np.float32)
+    guards = []
+    out = _guarded((B, C, s, s), torch.float32, guards)
+    xg = torch.from_numpy(x).cuda()
+    res = hmar.hmar_recon_downsample(xg, s, out=out)
+    assert res is out
+    ref = orc.area_downsample(x, s)
+    err = np.abs(out.double().cpu().numpy() - ref)
+    assert err.max() <= 1e-5 * max(1.0, np.abs(ref).max()), f"max abs err {err.max():.3e}"
+    assert torch.equal(xg.cpu(), torch.from_numpy(x))           # the input is read only
+    assert all(intact() for intact in guards)
+
+
 def test_recon_accumulate_codebook_off_16_byte_alignment():
     """A codebook whose base address is not a multiple of 16 bytes takes the staged kernel's one-value-at-a-time
     gather; same result as the oracle."""

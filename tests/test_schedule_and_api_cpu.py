@@ -152,6 +152,13 @@ def test_argument_errors_of_the_added_entry_points():
     assert g(p, p, None, p, p, None, 1, 32, 4096, 4, 32, None) == hmar.HMAR_ERR_BAD_ARG              # mask without old tokens
     assert g(p, p, p, p, p, p, 1, 32, 4096, 4, 32, None) == hmar.HMAR_ERR_BAD_ARG                    # tokens_out aliases an input
     assert g(p, p, None, p, None, None, 0, 32, 4096, 4, 32, None) == hmar.HMAR_ERR_BAD_ARG
+    d = L.hmar_recon_downsample
+    q2 = ctypes.c_void_p(p.value + 4096)
+    assert d(None, q2, 1, 32, 32, 13, None) == hmar.HMAR_ERR_BAD_ARG                                 # no input
+    assert d(p, None, 1, 32, 32, 13, None) == hmar.HMAR_ERR_BAD_ARG                                  # no output
+    assert d(p, p, 1, 32, 32, 13, None) == hmar.HMAR_ERR_BAD_ARG                                     # in place
+    assert d(p, q2, 1, 32, 13, 32, None) == hmar.HMAR_ERR_BAD_ARG                                    # would enlarge
+    assert d(p, q2, 1, 32, 32, 0, None) == hmar.HMAR_ERR_BAD_ARG
 
 
 def test_prev_window_backward_tiles_leave_out_nothing_but_the_last_scale():
