@@ -187,14 +187,25 @@ hmar_recon_accumulate_staged_kernel(float* __restrict__ xhat, const float* __res
 // one word); lane = input row sums the row's column bins (partial sums, row stride odd so the lanes hit
 // different banks); lane = output column sums those over the row bins, divides by the bin's size and writes
 // a coalesced output row.  One read of the reconstruction, which is all the traffic that counts.
+constexpr int kDownStageMaxSide = 64;
+constexpr size_t kDownStageSmem = 96 * 1024;
+
 __device__ __forceinline__ int bin_begin(int i, int in, int out) { return (i * in) / out; }
 __device__ __forceinline__ int bin_end(int i, int in, int out) { return ((i + 1) * in + out - 1) / out; }
 
+// SF: the input side as a compile-time constant (16, 32, 64: the latents of the paper's resolutions), so that a
+// lane's loads of the plane are all issued before the first is used -- a warp's 1 to 16 KB in flight is what brings
+// the read near the HBM rate; 0 = any side up to 64, eight loads at a time.
+template <int SF>
 __global__ void __launch_bounds__(256)
 hmar_recon_downsample_staged_kernel(const float* __restrict__ xhat, float* __restrict__ out, long long n_planes,
-                                    int S, int s, int warps_per_block) {
+                                    int S_any, int s, int warps_per_block) {
+    const int S = SF ? SF : S_any;
     extern __shared__ float down_smem[];
+    __shared__ int2 bins[kDownStageMaxSide];               // [begin, end) of every output index (rows and columns alike)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x < s) bins[threadIdx.x] = make_int2(bin_begin(threadIdx.x, S, s), bin_end(threadIdx.x, S, s));
+    __syncthreads();
     const int ts = s | 1;                                   // row stride of the partial sums
     const int per_warp = S * (S + 1) + S * ts;
     float* tile = down_smem + warp * per_warp;
@@ -202,29 +213,94 @@ hmar_recon_downsample_staged_kernel(const float* __restrict__ xhat, float* __res
     const long long plane = (long long)blockIdx.x * warps_per_block + warp;
     if (warp >= warps_per_block || plane >= n_planes) return;
     const float* src = xhat + plane * S * S;
-    for (int i = lane; i < S * S; i += 32) {
-        const int r = i / S, c = i - r * S;
-        tile[r * (S + 1) + c] = src[i];
-    }
-    __syncwarp();
-    for (int r = lane; r < S; r += 32) {
-        const float* row = tile + r * (S + 1);
-        for (int ox = 0; ox < s; ++ox) {
-            const int c0 = bin_begin(ox, S, s), c1 = bin_end(ox, S, s);
-            float acc = 0.f;
-            for (int c = c0; c < c1; ++c) acc += row[c];
-            part[r * ts + ox] = acc;
+    if (SF) {
+        constexpr int N = SF ? SF * SF / 32 : 1;           // values per lane
+        constexpr int CH = N < 32 ? N : 32;                // ... fetched CH at a time
+#pragma unroll 1
+        for (int i0 = 0; i0 < N; i0 += CH) {
+            float v[CH];
+#pragma unroll
+            for (int k = 0; k < CH; ++k) v[k] = src[(i0 + k) * 32 + lane];
+#pragma unroll
+            for (int k = 0; k < CH; ++k) {
+                const int i = (i0 + k) * 32 + lane, r = i / S, c = i - r * S;
+                tile[r * (S + 1) + c] = v[k];
+            }
+        }
+    } else {
+        const float inv = 1.f / (float)S;
+#pragma unroll 8
+        for (int i = lane; i < S * S; i += 32) {
+            const int r = (int)(((float)i + 0.5f) * inv), c = i - r * S;      // i / S: exact for i < 4096, S <= 64
+            tile[r * (S + 1) + c] = src[i];
         }
     }
     __syncwarp();
+    // Short bins (output side at least a third of the input side): four bins at a time, walked in step up to the
+    // longest bin's length with the shorter ones predicated off -- four independent chains of loads and additions
+    // per lane instead of one, since the sums are short and latency-bound.  Long bins: one after the other.
+    const int max_len = (S + s - 1) / s + 1;
+    const bool by_four = max_len <= 4;
     float* dst = out + plane * s * s;
-    for (int ox = lane; ox < s; ox += 32) {
-        const int nc = bin_end(ox, S, s) - bin_begin(ox, S, s);
-        for (int oy = 0; oy < s; ++oy) {
-            const int r0 = bin_begin(oy, S, s), r1 = bin_end(oy, S, s);
-            float acc = 0.f;
-            for (int r = r0; r < r1; ++r) acc += part[r * ts + ox];
-            dst[oy * s + ox] = acc / (float)((r1 - r0) * nc);
+    if (by_four) {
+        for (int r = lane; r < S; r += 32) {
+            const float* row = tile + r * (S + 1);
+            for (int ox = 0; ox < s; ox += 4) {
+                int2 cb[4];
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) cb[u] = ox + u < s ? bins[ox + u] : make_int2(0, 0);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (cb[u].x + k < cb[u].y) acc[u] += row[cb[u].x + k];
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (ox + u < s) part[r * ts + ox + u] = acc[u];
+            }
+        }
+        __syncwarp();
+        for (int ox = lane; ox < s; ox += 32) {
+            const int2 cbx = bins[ox];
+            const int nc = cbx.y - cbx.x;
+            for (int oy = 0; oy < s; oy += 4) {
+                int2 rb[4];
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) rb[u] = oy + u < s ? bins[oy + u] : make_int2(0, 0);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (rb[u].x + k < rb[u].y) acc[u] += part[(rb[u].x + k) * ts + ox];
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (oy + u < s) dst[(oy + u) * s + ox] = acc[u] / (float)((rb[u].y - rb[u].x) * nc);
+            }
+        }
+    } else {
+        for (int r = lane; r < S; r += 32) {
+            const float* row = tile + r * (S + 1);
+            for (int ox = 0; ox < s; ++ox) {
+                const int2 cb = bins[ox];
+                float acc = 0.f;
+                for (int c = cb.x; c < cb.y; ++c) acc += row[c];
+                part[r * ts + ox] = acc;
+            }
+        }
+        __syncwarp();
+        for (int ox = lane; ox < s; ox += 32) {
+            const int2 cb = bins[ox];
+            const int nc = cb.y - cb.x;
+            for (int oy = 0; oy < s; ++oy) {
+                const int2 rb = bins[oy];
+                float acc = 0.f;
+                for (int r = rb.x; r < rb.y; ++r) acc += part[r * ts + ox];
+                dst[oy * s + ox] = acc / (float)((rb.y - rb.x) * nc);
+            }
         }
     }
 }
@@ -273,8 +349,6 @@ cudaError_t launch_recon_accumulate(float* xhat, const float* codebook, const in
     return cudaGetLastError();
 }
 
-constexpr int kDownStageMaxSide = 64;
-constexpr size_t kDownStageSmem = 96 * 1024;
 
 cudaError_t launch_recon_downsample(const float* xhat, float* out, int B, int C, int in_side, int out_side,
                                     cudaStream_t stream) {
@@ -284,14 +358,18 @@ cudaError_t launch_recon_downsample(const float* xhat, float* out, int B, int C,
         int warps = (int)(kDownStageSmem / per_warp);
         warps = warps > 8 ? 8 : warps;                      // >= 2 at the largest staged plane
         const size_t smem = per_warp * warps;
-        cudaError_t e = cudaFuncSetAttribute(hmar_recon_downsample_staged_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)kDownStageSmem);
+        const unsigned grid = (unsigned)((n_planes + warps - 1) / warps);
+        cudaError_t e = cudaSuccess;
+        KernelTimer timer("hmar_recon_downsample_kernel", stream);
+        auto go = [&](auto kernel) {
+            e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDownStageSmem);
+            if (e == cudaSuccess) kernel<<<grid, 256, smem, stream>>>(xhat, out, n_planes, in_side, out_side, warps);
+        };
+        if (in_side == 16) go(hmar_recon_downsample_staged_kernel<16>);
+        else if (in_side == 32) go(hmar_recon_downsample_staged_kernel<32>);
+        else if (in_side == 64) go(hmar_recon_downsample_staged_kernel<64>);
+        else go(hmar_recon_downsample_staged_kernel<0>);
         if (e != cudaSuccess) return e;
-        {
-            KernelTimer timer("hmar_recon_downsample_kernel", stream);
-            hmar_recon_downsample_staged_kernel<<<(unsigned)((n_planes + warps - 1) / warps), 256, smem, stream>>>(
-                xhat, out, n_planes, in_side, out_side, warps);
-        }
         count_launch(1);
         return cudaGetLastError();
     }
