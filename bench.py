@@ -677,7 +677,8 @@ def run_case(args):
     """A named side case run a few times (for profiling one kernel on a workload that is not the headline's):
     `256_d30_train` = forward + backward of the L = 680 training config at its full batch; `infer_scale7` = the
     inference step of scale 7 (169 queries, 250 keys) at B = 64, H = 24; `recon_b2048` = the sampler's neighbour step
-    on a 32 x 32 x 32 reconstruction at B = 2048 (268 MB), a 13 x 13 map then the 32 x 32 one per repetition.
+    on a 32 x 32 x 32 reconstruction at B = 2048 (268 MB), a 13 x 13 map then the 32 x 32 one per repetition, each
+    followed by the area interpolation down to 13 x 13 and to 32 x 32.
     Prints a small JSON line."""
     import torch
 
@@ -707,6 +708,8 @@ def run_case(args):
             for side in (13, 32):
                 new, old, mask, sel = maps[side]
                 hmar.hmar_recon_accumulate(xhat, codebook, new, old, mask, sel)
+            for side in (13, 32):
+                hmar.hmar_recon_downsample(xhat, side)
     else:
         wl_x = CONFIGS["512_d24_infer"]
         s_ = 6

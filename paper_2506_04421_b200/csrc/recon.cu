@@ -186,7 +186,8 @@ hmar_recon_accumulate_staged_kernel(float* __restrict__ xhat, const float* __res
 // Staged kernel: a warp per image plane.  The plane is read once, coalesced, into shared memory (rows padded by
 // one word); lane = input row sums the row's column bins (partial sums, row stride odd so the lanes hit
 // different banks); lane = output column sums those over the row bins, divides by the bin's size and writes
-// a coalesced output row.  One read of the reconstruction, which is all the traffic that counts.
+// a coalesced output row.  One read of the reconstruction, which is all the traffic that counts.  Equal sizes are
+// a plain copy (the launcher does it).
 constexpr int kDownStageMaxSide = 64;
 constexpr size_t kDownStageSmem = 96 * 1024;
 
@@ -204,10 +205,10 @@ hmar_recon_downsample_staged_kernel(const float* __restrict__ xhat, float* __res
     extern __shared__ float down_smem[];
     __shared__ int2 bins[kDownStageMaxSide];               // [begin, end) of every output index (rows and columns alike)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x < s) bins[threadIdx.x] = make_int2(bin_begin(threadIdx.x, S, s), bin_end(threadIdx.x, S, s));
+    for (int i = threadIdx.x; i < s; i += blockDim.x) bins[i] = make_int2(bin_begin(i, S, s), bin_end(i, S, s));
     __syncthreads();
     const int ts = s | 1;                                   // row stride of the partial sums
-    const int per_warp = S * (S + 1) + S * ts;
+    const int per_warp = S * (S + 1) + (S + 1) * ts;
     float* tile = down_smem + warp * per_warp;
     float* part = tile + S * (S + 1);
     const long long plane = (long long)blockIdx.x * warps_per_block + warp;
@@ -236,71 +237,73 @@ hmar_recon_downsample_staged_kernel(const float* __restrict__ xhat, float* __res
         }
     }
     __syncwarp();
-    // Short bins (output side at least a third of the input side): four bins at a time, walked in step up to the
-    // longest bin's length with the shorter ones predicated off -- four independent chains of loads and additions
-    // per lane instead of one, since the sums are short and latency-bound.  Long bins: one after the other.
-    const int max_len = (S + s - 1) / s + 1;
-    const bool by_four = max_len <= 4;
-    float* dst = out + plane * s * s;
-    if (by_four) {
-        for (int r = lane; r < S; r += 32) {
-            const float* row = tile + r * (S + 1);
-            for (int ox = 0; ox < s; ox += 4) {
-                int2 cb[4];
-                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float* dst0 = out + plane * s * s;
+    if (SF) {
+        // Compile-time side: running sums.  Lane = input row turns its row into exclusive running sums in place (the
+        // padded row has exactly S + 1 slots), so a column bin's sum is one difference; lane = output column does the
+        // same down the partial sums' columns.  Everything is straight-line code over registers, and the loops over
+        // the bins have independent iterations.
+        constexpr int SS = SF ? SF : 1;
+        for (int r = lane; r < SS; r += 32) {
+            float* row = tile + r * (SS + 1);
+            float v[SS];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) cb[u] = ox + u < s ? bins[ox + u] : make_int2(0, 0);
+            for (int c = 0; c < SS; ++c) v[c] = row[c];
+            float run = 0.f;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (cb[u].x + k < cb[u].y) acc[u] += row[cb[u].x + k];
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (ox + u < s) part[r * ts + ox + u] = acc[u];
+            for (int c = 0; c < SS; ++c) {
+                row[c] = run;
+                run += v[c];
+            }
+            row[SS] = run;
+#pragma unroll 4
+            for (int ox = 0; ox < s; ++ox) {
+                const int2 cb = bins[ox];
+                part[r * ts + ox] = row[cb.y] - row[cb.x];
             }
         }
         __syncwarp();
         for (int ox = lane; ox < s; ox += 32) {
             const int2 cbx = bins[ox];
             const int nc = cbx.y - cbx.x;
-            for (int oy = 0; oy < s; oy += 4) {
-                int2 rb[4];
-                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            float* col = part + ox;
+            float v[SS];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) rb[u] = oy + u < s ? bins[oy + u] : make_int2(0, 0);
+            for (int r = 0; r < SS; ++r) v[r] = col[r * ts];
+            float run = 0.f;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (rb[u].x + k < rb[u].y) acc[u] += part[(rb[u].x + k) * ts + ox];
-                }
-#pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (oy + u < s) dst[(oy + u) * s + ox] = acc[u] / (float)((rb[u].y - rb[u].x) * nc);
+            for (int r = 0; r < SS; ++r) {
+                col[r * ts] = run;
+                run += v[r];
             }
-        }
-    } else {
-        for (int r = lane; r < S; r += 32) {
-            const float* row = tile + r * (S + 1);
-            for (int ox = 0; ox < s; ++ox) {
-                const int2 cb = bins[ox];
-                float acc = 0.f;
-                for (int c = cb.x; c < cb.y; ++c) acc += row[c];
-                part[r * ts + ox] = acc;
-            }
-        }
-        __syncwarp();
-        for (int ox = lane; ox < s; ox += 32) {
-            const int2 cb = bins[ox];
-            const int nc = cb.y - cb.x;
+            col[SS * ts] = run;
+#pragma unroll 4
             for (int oy = 0; oy < s; ++oy) {
                 const int2 rb = bins[oy];
-                float acc = 0.f;
-                for (int r = rb.x; r < rb.y; ++r) acc += part[r * ts + ox];
-                dst[oy * s + ox] = acc / (float)((rb.y - rb.x) * nc);
+                dst0[oy * s + ox] = (col[rb.y * ts] - col[rb.x * ts]) / (float)((rb.y - rb.x) * nc);
             }
+        }
+        return;
+    }
+    // Any other side: the bins one after the other.
+    for (int r = lane; r < S; r += 32) {
+        const float* row = tile + r * (S + 1);
+        for (int ox = 0; ox < s; ++ox) {
+            const int2 cb = bins[ox];
+            float acc = 0.f;
+            for (int c = cb.x; c < cb.y; ++c) acc += row[c];
+            part[r * ts + ox] = acc;
+        }
+    }
+    __syncwarp();
+    for (int ox = lane; ox < s; ox += 32) {
+        const int2 cb = bins[ox];
+        const int nc = cb.y - cb.x;
+        for (int oy = 0; oy < s; ++oy) {
+            const int2 rb = bins[oy];
+            float acc = 0.f;
+            for (int r = rb.x; r < rb.y; ++r) acc += part[r * ts + ox];
+            dst0[oy * s + ox] = acc / (float)((rb.y - rb.x) * nc);
         }
     }
 }
@@ -353,8 +356,11 @@ cudaError_t launch_recon_accumulate(float* xhat, const float* codebook, const in
 cudaError_t launch_recon_downsample(const float* xhat, float* out, int B, int C, int in_side, int out_side,
                                     cudaStream_t stream) {
     const long long n_planes = (long long)B * C;
+    if (in_side == out_side) {                              // every bin is one pixel: a copy, bit for bit
+        return cudaMemcpyAsync(out, xhat, (size_t)n_planes * in_side * in_side * sizeof(float), cudaMemcpyDeviceToDevice, stream);
+    }
     if (in_side <= kDownStageMaxSide) {
-        const size_t per_warp = ((size_t)in_side * (in_side + 1) + (size_t)in_side * (out_side | 1)) * sizeof(float);
+        const size_t per_warp = ((size_t)in_side * (in_side + 1) + (size_t)(in_side + 1) * (out_side | 1)) * sizeof(float);
         int warps = (int)(kDownStageSmem / per_warp);
         warps = warps > 8 ? 8 : warps;                      // >= 2 at the largest staged plane
         const size_t smem = per_warp * warps;
@@ -363,7 +369,7 @@ cudaError_t launch_recon_downsample(const float* xhat, float* out, int B, int C,
         KernelTimer timer("hmar_recon_downsample_kernel", stream);
         auto go = [&](auto kernel) {
             e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDownStageSmem);
-            if (e == cudaSuccess) kernel<<<grid, 256, smem, stream>>>(xhat, out, n_planes, in_side, out_side, warps);
+            if (e == cudaSuccess) kernel<<<grid, warps * 32, smem, stream>>>(xhat, out, n_planes, in_side, out_side, warps);
         };
         if (in_side == 16) go(hmar_recon_downsample_staged_kernel<16>);
         else if (in_side == 32) go(hmar_recon_downsample_staged_kernel<32>);
