@@ -222,7 +222,8 @@ int hmar_recon_accumulate(float* xhat, const float* codebook, const int* tokens_
  * interpolation: out(i, j) = the mean of xhat over rows [floor(i * in_side / out_side),
  * ceil((i + 1) * in_side / out_side)) and the like columns.
  *   xhat : [B, C, in_side, in_side] fp32, device (read only);  out : [B, C, out_side, out_side] fp32, device
- * out_side <= in_side <= 4096; the buffers must not overlap.  One kernel, asynchronous on `stream`. */
+ * out_side <= in_side <= 4096; the buffers must not overlap.  One kernel (a device-to-device copy when the sizes
+ * are equal), asynchronous on `stream`. */
 int hmar_recon_downsample(const float* xhat, float* out, int B, int C, int in_side, int out_side, void* stream);
 
 /* Host-side scale-block scheduler (Sec. 4.1: the kernel visits only the live blocks of the mask).
